@@ -58,8 +58,23 @@ typedef enum {
     SPECV_ERR_WORKSPACE = 5,  /* workspace or arena smaller than required */
     SPECV_ERR_CUDA = 6,       /* a CUDA call failed; see spec_verify_last_cuda_error */
     SPECV_ERR_ARCH = 7,       /* the current device is not compute capability 10.x */
-    SPECV_ERR_TOO_LARGE = 8   /* spec_verify_noalloc only: batch exceeds the built-in scratch */
+    SPECV_ERR_TOO_LARGE = 8,  /* spec_verify_noalloc only: batch exceeds the built-in scratch */
+    SPECV_ERR_FLAGS = 9       /* unknown flag bits, both kernel-set bits, or a flag the call does not take */
 } specv_status;
+
+/* Per-call options (`flags` arguments).  The library keeps no mode between calls: two host threads
+ * may run passes with different options at the same time (on different workspaces). */
+enum {
+    SPECV_FLAG_STREAMING = 1,   /* use the streaming kernels (any shape) */
+    SPECV_FLAG_RING = 2,        /* use the ring kernels (bulk async copies into a shared-memory ring, the
+                                   batch cut into equal byte ranges per SM) whenever the shape allows them:
+                                   rows on 16-byte boundaries, V*elt a multiple of 16, V at most 2^19
+                                   elements for bf16 / fp16 and 2^18 for fp32, at most 4095 sequences;
+                                   else streaming.  Neither bit: automatic, the ring kernels from 64
+                                   target rows up.  Results of the two sets agree except for draws within
+                                   rounding of a decision boundary. */
+    SPECV_FLAG_EARLY_EXIT = 4   /* spec_verify_ex only; see there */
+};
 
 /* Bits of row_status[b] (data errors found on the device; the call itself succeeds).
  * With any of the first three set the sequence yields accepted_len 0 and -1 tokens. */
@@ -139,30 +154,39 @@ int spec_verify(const void* target_logits, const void* draft_logits, int dtype,
                 void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Kernel-set choice for later spec_verify calls of this process: 0 = automatic (default),
- * 1 = always the streaming kernels (any shape), 2 = the ring kernels (bulk async copies into a
- * shared-memory ring; the batch cut into equal byte ranges per SM) whenever the shape allows
- * them -- rows on 16-byte boundaries, V*elt a multiple of 16, V at most 2^19 elements for bf16 /
- * fp16 and 2^18 for fp32, at most 4095 sequences -- else streaming.  Automatic takes the ring
- * kernels from 64 target rows up.  Results of the two sets agree except for draws within rounding
- * of a decision boundary.  Returns SPECV_ERR_SHAPE for any other value.
+ * spec_verify with per-call options and, optionally, the lookahead of the next speculation round
+ * written by the same kernels.  spec_verify(...) is spec_verify_ex(..., 0, 0, 0, NULL).
+ *
+ *   flags   SPECV_FLAG_STREAMING or SPECV_FLAG_RING (kernel set; neither: automatic), and
+ *           SPECV_FLAG_EARLY_EXIT: the paper's theme is to do only the work the input needs; in this
+ *           pass nothing after a sequence's first rejected draft token can be emitted, so the logits
+ *           rows of later positions need not be read.  With this flag the ring kernels process the
+ *           positions of all sequences in order (position 0 of every sequence first) and skip every
+ *           row pair that lies after a position already rejected with a clear margin.  accepted_len,
+ *           emitted_tokens and row_status are exactly those of the normal mode; diag_p_tok /
+ *           diag_q_tok are NaN at skipped positions.  Ignored whenever the streaming kernels run.
+ *   next_k  device out, int32 [B], may be NULL: the lookahead for the next round (the paper's
+ *           input-dependent speculation, sections "Dynamic Execution" and "Speculative Sampling
+ *           Results"; the paper gives no rule, this is a stated heuristic): K_b + 2 if every drafted
+ *           token of sequence b was accepted, else K_b - 1, clamped to [k_min, k_max]; for a sequence
+ *           with a data error accepted_len counts as 0 and a negative K_b as 0.  Written by the warp
+ *           that emits the sequence's tokens; it never influences which tokens are emitted.
+ *   k_min, k_max   used only with next_k: 0 <= k_min <= k_max, else SPECV_ERR_SHAPE.
+ * Unknown flag bits or both kernel-set bits: SPECV_ERR_FLAGS.  Everything else as for spec_verify.
  */
-int spec_verify_set_path(int path);
+int spec_verify_ex(const void* target_logits, const void* draft_logits, int dtype,
+                   int64_t V, int64_t ld_target, int64_t ld_draft,
+                   const int32_t* draft_tokens, const int32_t* k_per_row,
+                   int32_t B, int32_t k_uniform, int64_t n_draft_total,
+                   const float* temperature, int temperature_per_row,
+                   const float* uniforms,
+                   int32_t* accepted_len, int32_t* emitted_tokens, int32_t* row_status,
+                   float* diag_p_tok, float* diag_q_tok,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream,
+                   uint32_t flags, int32_t k_min, int32_t k_max, int32_t* next_k);
 
-/*
- * Early exit (off by default).  The paper's theme is to do only the work the input needs; in
- * this pass nothing after a sequence's first rejected draft token can be emitted, so the logits
- * rows of later positions need not be read.  With enable != 0 the ring kernels process the
- * positions of all sequences in order (position 0 of every sequence first) and skip every row
- * pair that lies after a position already rejected with a clear margin.  accepted_len,
- * emitted_tokens and row_status are exactly those of the normal mode; diag_p_tok / diag_q_tok
- * are NaN at skipped positions.  Ignored (normal mode) whenever the streaming kernels run.
- * Always returns SPECV_OK.
- */
-int spec_verify_set_early_exit(int enable);
-
-/* Kernel set the calling thread's most recent spec_verify call used: 1 streaming, 2 ring,
- * 0 if it has made none.  Not a status code. */
+/* Kernel set the calling thread's most recent pass (any entry point below or above) used:
+ * 1 streaming, 2 ring, 0 if it has made none.  Not a status code. */
 int spec_verify_last_path(void);
 
 /*
@@ -183,7 +207,8 @@ int spec_verify_set_trace_events(void* const* events);
  * stated heuristic): next_k[b] = K_b + 2 if every drafted token of sequence b was accepted
  * (accepted_len[b] >= K_b), else K_b - 1, clamped to [k_min, k_max].  It never influences
  * which tokens are emitted.  k_per_row (or NULL with k_uniform), accepted_len and next_k are
- * DEVICE int32 arrays of B entries; one small kernel is enqueued on cuda_stream.  Returns
+ * DEVICE int32 arrays of B entries; one small kernel is enqueued on cuda_stream (spec_verify_ex can
+ * write the same values from inside the pass, without this extra launch).  Returns
  * SPECV_ERR_NULL / SPECV_ERR_SHAPE (B < 1, k_min < 0, k_max < k_min) / SPECV_ERR_CUDA.
  */
 int spec_verify_next_lookahead(const int32_t* k_per_row, int32_t k_uniform, const int32_t* accepted_len,
@@ -225,8 +250,10 @@ int spec_verify_next_lookahead(const int32_t* k_per_row, int32_t k_uniform, cons
  *   diag_p_tok, diag_q_tok [n_node_total], may be NULL  p_c(x_j), q_c(x_j) of EVERY node j, c the
  *                                                 context of its parent
  *   workspace                                     >= spec_verify_tree_workspace_bytes(B, n_node_total, V)
+ *   flags                                         SPECV_FLAG_STREAMING / SPECV_FLAG_RING or 0 (kernel set of
+ *                                                 the row statistics); SPECV_FLAG_EARLY_EXIT is refused
  * Everything else (pointers are DEVICE pointers, dtype, temperature, row_status, asynchrony, error
- * reporting, spec_verify_set_path) as for spec_verify.  Each rejected child costs one more pass
+ * reporting) as for spec_verify.  Each rejected child costs one more pass
  * over its context's two rows; the row statistics are computed once for every row that is needed.
  */
 size_t spec_verify_tree_workspace_bytes(int32_t B, int64_t n_node_total, int64_t V);
@@ -237,7 +264,7 @@ int spec_verify_tree(const void* target_logits, const void* draft_logits, int dt
                      const float* temperature, int temperature_per_seq, const float* uniforms,
                      int32_t* accepted_len, int32_t* emitted_tokens, int32_t* accepted_nodes,
                      int32_t* row_status, float* diag_p_tok, float* diag_q_tok,
-                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+                     void* workspace, size_t workspace_bytes, void* cuda_stream, uint32_t flags);
 
 /*
  * Greedy verification: the temperature -> 0 limit of the pass above (the paper's section
@@ -260,8 +287,9 @@ int spec_verify_tree(const void* target_logits, const void* draft_logits, int dt
  *   workspace, workspace_bytes device scratch, 256-byte aligned,
  *                              >= spec_verify_greedy_workspace_bytes(B, n_draft_total); need not
  *                              be initialised, clobbered
- * spec_verify_set_path applies: the ring kernel (bulk async copies) needs rows on 16-byte
- * boundaries with V*elt a multiple of 16 and is chosen automatically from 64 target rows up.
+ *   flags                      SPECV_FLAG_STREAMING / SPECV_FLAG_RING or 0: the ring kernel (bulk async
+ *                              copies) needs rows on 16-byte boundaries with V*elt a multiple of 16 and
+ *                              is chosen automatically from 64 target rows up
  */
 size_t spec_verify_greedy_workspace_bytes(int32_t B, int64_t n_draft_total);
 int spec_verify_greedy(const void* target_logits, int dtype, int64_t V, int64_t ld_target,
@@ -269,7 +297,7 @@ int spec_verify_greedy(const void* target_logits, int dtype, int64_t V, int64_t 
                        int32_t B, int32_t k_uniform, int64_t n_draft_total,
                        int32_t* accepted_len, int32_t* emitted_tokens, int32_t* row_status,
                        int32_t* target_argmax,
-                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+                       void* workspace, size_t workspace_bytes, void* cuda_stream, uint32_t flags);
 
 /*
  * Bytes of device memory ("arena") that spec_verify_host needs: device copies of all
@@ -313,8 +341,9 @@ int spec_verify_host(const void* target_logits, const void* draft_logits, int dt
  * no allocation of any kind (no cudaMalloc/cudaFree, no allocating library routine).
  *
  * Arguments, layout, outputs, asynchrony and error reporting are exactly those of
- * spec_verify, without `workspace` / `workspace_bytes`; results are identical to spec_verify's.
- * Differences:
+ * spec_verify, without `workspace` / `workspace_bytes`.  The same kernels run as for spec_verify on
+ * the same batch (same automatic choice of the kernel set), so the results are bit-identical to
+ * spec_verify's.  Differences:
  *   - Size limit: spec_verify_workspace_bytes(B, n_draft_total, V) must not exceed
  *     SPECV_NOALLOC_SCRATCH_BYTES (4 MiB -- e.g. 64 sequences x 8 drafts over a vocabulary of
  *     128256 need 0.3 MiB, 256 x 4 over 152064 need 1.3 MiB; the size grows with B * V);
@@ -322,8 +351,8 @@ int spec_verify_host(const void* target_logits, const void* draft_logits, int dt
  *   - First call on each device looks up the array's device address (once per device, with
  *     that device current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left
- *     in it.  Nothing in it needs to be zero on entry (each call writes every word before
- *     reading it), but two calls whose kernels overlap on the GPU -- different streams, or
+ *     in it.  Nothing in it needs to be zero on entry (each call writes every word, the tickets
+ *     and counters that must start at zero included, before reading it), but two calls whose kernels overlap on the GPU -- different streams, or
  *     different host threads -- would overwrite each other's scratch: serialise them (same
  *     stream, or an event between them).
  */

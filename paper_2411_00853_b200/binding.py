@@ -21,7 +21,8 @@ ROW_INTERNAL, ROW_BAD_PARENT = 16, 32
 
 EXPORTS = ("spec_verify", "spec_verify_host", "spec_verify_workspace_bytes",
            "spec_verify_host_arena_bytes", "spec_verify_strerror", "spec_verify_last_cuda_error",
-           "spec_verify_launch_count", "spec_verify_set_trace_events", "spec_verify_noalloc", "spec_verify_set_path", "spec_verify_last_path", "spec_verify_set_early_exit", "spec_verify_next_lookahead",
+           "spec_verify_launch_count", "spec_verify_set_trace_events", "spec_verify_noalloc", "spec_verify_ex",
+           "spec_verify_last_path", "spec_verify_next_lookahead",
            "spec_verify_greedy", "spec_verify_greedy_workspace_bytes",
            "spec_verify_tree", "spec_verify_tree_workspace_bytes")
 NOALLOC_SCRATCH_BYTES = 4 << 20
@@ -54,23 +55,22 @@ def load() -> ctypes.CDLL:
     lib.spec_verify_host.argtypes = common
     lib.spec_verify_noalloc.restype = ctypes.c_int
     lib.spec_verify_noalloc.argtypes = common[:-3] + [vp]
-    lib.spec_verify_set_early_exit.restype = ctypes.c_int
-    lib.spec_verify_set_early_exit.argtypes = [ctypes.c_int]
+    lib.spec_verify_ex.restype = ctypes.c_int
+    lib.spec_verify_ex.argtypes = common + [ctypes.c_uint32, i32, i32, vp]
     lib.spec_verify_next_lookahead.restype = ctypes.c_int
     lib.spec_verify_next_lookahead.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp]
     lib.spec_verify_tree.restype = ctypes.c_int
     lib.spec_verify_tree.argtypes = [vp, vp, ctypes.c_int, i64, i64, i64, vp, vp, vp, i32, i32, i64, vp, ctypes.c_int,
-                                     vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+                                     vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, ctypes.c_uint32]
     lib.spec_verify_tree_workspace_bytes.restype = sz
     lib.spec_verify_tree_workspace_bytes.argtypes = [i32, i64, i64]
     lib.spec_verify_greedy.restype = ctypes.c_int
-    lib.spec_verify_greedy.argtypes = [vp, ctypes.c_int, i64, i64, vp, vp, i32, i32, i64, vp, vp, vp, vp, vp, sz, vp]
+    lib.spec_verify_greedy.argtypes = [vp, ctypes.c_int, i64, i64, vp, vp, i32, i32, i64, vp, vp, vp, vp, vp, sz, vp,
+                                       ctypes.c_uint32]
     lib.spec_verify_greedy_workspace_bytes.restype = sz
     lib.spec_verify_greedy_workspace_bytes.argtypes = [i32, i64]
     lib.spec_verify_last_path.restype = ctypes.c_int
     lib.spec_verify_last_path.argtypes = []
-    lib.spec_verify_set_path.restype = ctypes.c_int
-    lib.spec_verify_set_path.argtypes = [ctypes.c_int]
     lib.spec_verify_workspace_bytes.restype = sz
     lib.spec_verify_workspace_bytes.argtypes = [i32, i64, i64]
     lib.spec_verify_host_arena_bytes.restype = sz
@@ -112,16 +112,31 @@ def set_trace_events(events):
 
 
 PATH_AUTO, PATH_STREAMING, PATH_RING = 0, 1, 2
+FLAG_STREAMING, FLAG_RING, FLAG_EARLY_EXIT = 1, 2, 4
+
+# The C library keeps no mode between calls: options travel with every call as `flags`.  For
+# convenience (tests, the benchmark) this module holds DEFAULT flags that its wrappers pass when
+# the caller gives none; they are plain Python state of this module, not of the library.
+_default_flags = 0
 
 
 def set_path(path: int):
-    """Kernel-set choice for later calls: PATH_AUTO, PATH_STREAMING or PATH_RING."""
-    _check(load().spec_verify_set_path(path))
+    """Default kernel set of this module's wrappers: PATH_AUTO, PATH_STREAMING or PATH_RING."""
+    global _default_flags
+    if path not in (PATH_AUTO, PATH_STREAMING, PATH_RING):
+        raise ValueError("path must be PATH_AUTO, PATH_STREAMING or PATH_RING")
+    _default_flags = (_default_flags & ~(FLAG_STREAMING | FLAG_RING)) | path
 
 
 def set_early_exit(enable: bool):
-    """Skip logits rows after a sequence's first clear rejection (ring kernels only; same tokens)."""
-    _check(load().spec_verify_set_early_exit(int(bool(enable))))
+    """Default of this module's spec_verify wrapper: skip logits rows after a sequence's first
+    clear rejection (ring kernels only; same tokens)."""
+    global _default_flags
+    _default_flags = (_default_flags | FLAG_EARLY_EXIT) if enable else (_default_flags & ~FLAG_EARLY_EXIT)
+
+
+def default_flags() -> int:
+    return _default_flags
 
 
 def next_lookahead(k_per_row, accepted_len, k_min: int, k_max: int, *, k_uniform: int = 0, out=None, stream=None):
@@ -163,6 +178,16 @@ def _ptr(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
 
 
+def _temporary_workspace(nbytes: int, dev, stream):
+    """Scratch allocated for one call.  When the call runs on a caller-given raw stream, torch's
+    allocator is told that the block is in use there, so it is not handed out again before the
+    pass has finished."""
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=dev)
+    if stream is not None:
+        ws.record_stream(torch.cuda.ExternalStream(int(stream), device=dev))
+    return ws
+
+
 def _shape_args(target_logits, draft_logits, k_per_row, k_uniform):
     assert target_logits.dim() == 2 and target_logits.stride(1) == 1
     V = target_logits.shape[1]
@@ -184,15 +209,19 @@ def _shape_args(target_logits, draft_logits, k_per_row, k_uniform):
 
 def spec_verify(target_logits, draft_logits, draft_tokens, k_per_row, temperature, uniforms, *,
                 k_uniform=None, accepted_len=None, emitted_tokens=None, row_status=None,
-                diag_p_tok=None, diag_q_tok=None, workspace=None, stream=None):
-    """Enqueue one verify-and-resample pass on CUDA tensors (see include/spec_verify.h).
+                diag_p_tok=None, diag_q_tok=None, workspace=None, stream=None, flags=None,
+                next_k=None, k_min=0, k_max=0):
+    """Enqueue one verify-and-resample pass on CUDA tensors (spec_verify_ex of include/spec_verify.h).
 
     target_logits [sum(K)+B, V], draft_logits [sum(K), V]: float32 or bfloat16, row pitch = stride(0)
     draft_tokens int32 [sum(K)], k_per_row int32 [B] or None (then every sequence has k_uniform drafts)
     temperature float32 [1] or [B], uniforms float32 [sum(K)+B]
     Returns (accepted_len int32 [B], emitted_tokens int32 [sum(K)+B]); the call is asynchronous
     on `stream` (default: torch's current stream).  Output / scratch tensors may be passed in to
-    avoid allocations.
+    avoid allocations.  flags: FLAG_* bits (default: this module's default flags); next_k: int32 [B]
+    CUDA tensor that receives the next round's lookahead, clamped to [k_min, k_max].
+    With a `stream` other than torch's current one, pass a `workspace` you own: a temporary
+    allocated here would be returned to torch's allocator while the pass may still be running.
     """
     lib = load()
     dev = target_logits.device
@@ -204,14 +233,15 @@ def spec_verify(target_logits, draft_logits, draft_tokens, k_per_row, temperatur
         emitted_tokens = torch.empty(D + B, dtype=torch.int32, device=dev)
     need = workspace_bytes(B, D, V)
     if workspace is None:
-        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        workspace = _temporary_workspace(need, dev, stream)
     if stream is None:
         stream = torch.cuda.current_stream(dev).cuda_stream
-    rc = lib.spec_verify(_ptr(target_logits), _ptr(draft_logits) if D else None, _dtype_code(target_logits),
-                         V, ld_t, ld_d, _ptr(draft_tokens) if D else None, _ptr(k_per_row), B, k_uniform, D,
-                         _ptr(temperature), per_row, _ptr(uniforms), _ptr(accepted_len), _ptr(emitted_tokens),
-                         _ptr(row_status), _ptr(diag_p_tok), _ptr(diag_q_tok), _ptr(workspace),
-                         workspace.numel() * workspace.element_size(), ctypes.c_void_p(stream))
+    rc = lib.spec_verify_ex(_ptr(target_logits), _ptr(draft_logits) if D else None, _dtype_code(target_logits),
+                            V, ld_t, ld_d, _ptr(draft_tokens) if D else None, _ptr(k_per_row), B, k_uniform, D,
+                            _ptr(temperature), per_row, _ptr(uniforms), _ptr(accepted_len), _ptr(emitted_tokens),
+                            _ptr(row_status), _ptr(diag_p_tok), _ptr(diag_q_tok), _ptr(workspace),
+                            workspace.numel() * workspace.element_size(), ctypes.c_void_p(stream),
+                            _default_flags if flags is None else int(flags), int(k_min), int(k_max), _ptr(next_k))
     _check(rc)
     return accepted_len, emitted_tokens
 
@@ -260,12 +290,18 @@ def spec_verify_host(target_logits, draft_logits, draft_tokens, k_per_row, tempe
     return accepted_len, emitted_tokens
 
 
+def _path_flags(flags) -> int:
+    """Flags for the entry points that take a kernel-set choice only."""
+    return (_default_flags if flags is None else int(flags)) & (FLAG_STREAMING | FLAG_RING)
+
+
 def greedy_workspace_bytes(B: int, n_draft_total: int) -> int:
     return int(load().spec_verify_greedy_workspace_bytes(B, n_draft_total))
 
 
 def spec_verify_greedy(target_logits, draft_tokens, k_per_row, *, k_uniform=None, accepted_len=None,
-                       emitted_tokens=None, row_status=None, target_argmax=None, workspace=None, stream=None):
+                       emitted_tokens=None, row_status=None, target_argmax=None, workspace=None, stream=None,
+                       flags=None):
     """Enqueue one greedy verification pass (temperature -> 0: accept while the draft token is the
     target row's argmax) on CUDA tensors.  target_logits [sum(K)+B, V]; draft_tokens int32 [sum(K)];
     k_per_row int32 [B] or None with k_uniform.  Returns (accepted_len, emitted_tokens)."""
@@ -285,14 +321,14 @@ def spec_verify_greedy(target_logits, draft_tokens, k_per_row, *, k_uniform=None
     if emitted_tokens is None:
         emitted_tokens = torch.empty(D + B, dtype=torch.int32, device=dev)
     if workspace is None:
-        workspace = torch.empty(max(greedy_workspace_bytes(B, D), 256), dtype=torch.uint8, device=dev)
+        workspace = _temporary_workspace(greedy_workspace_bytes(B, D), dev, stream)
     if stream is None:
         stream = torch.cuda.current_stream(dev).cuda_stream
     rc = lib.spec_verify_greedy(_ptr(target_logits), _dtype_code(target_logits), V, ld_t,
                                 _ptr(draft_tokens) if D else None, _ptr(k_per_row), B, int(k_uniform), D,
                                 _ptr(accepted_len), _ptr(emitted_tokens), _ptr(row_status), _ptr(target_argmax),
                                 _ptr(workspace), workspace.numel() * workspace.element_size(),
-                                ctypes.c_void_p(stream))
+                                ctypes.c_void_p(stream), _path_flags(flags))
     _check(rc)
     return accepted_len, emitted_tokens
 
@@ -303,7 +339,7 @@ def tree_workspace_bytes(B: int, n_node_total: int, V: int) -> int:
 
 def spec_verify_tree(target_logits, draft_logits, node_tokens, node_parent, n_per_seq, temperature, uniforms, *,
                      n_uniform=None, accepted_len=None, emitted_tokens=None, accepted_nodes=None, row_status=None,
-                     diag_p_tok=None, diag_q_tok=None, workspace=None, stream=None):
+                     diag_p_tok=None, diag_q_tok=None, workspace=None, stream=None, flags=None):
     """Enqueue one tree-structured verification pass on CUDA tensors (see include/spec_verify.h).
     target_logits [sum(N)+B, V] (row of context c), draft_logits [sum(N), V], node_tokens / node_parent
     int32 [sum(N)], n_per_seq int32 [B] (or None with n_uniform).  Returns (accepted_len, emitted_tokens)."""
@@ -316,7 +352,7 @@ def spec_verify_tree(target_logits, draft_logits, node_tokens, node_parent, n_pe
     if emitted_tokens is None:
         emitted_tokens = torch.empty(D + B, dtype=torch.int32, device=dev)
     if workspace is None:
-        workspace = torch.empty(max(tree_workspace_bytes(B, D, V), 256), dtype=torch.uint8, device=dev)
+        workspace = _temporary_workspace(tree_workspace_bytes(B, D, V), dev, stream)
     if stream is None:
         stream = torch.cuda.current_stream(dev).cuda_stream
     rc = lib.spec_verify_tree(_ptr(target_logits), _ptr(draft_logits) if D else None, _dtype_code(target_logits),
@@ -324,6 +360,7 @@ def spec_verify_tree(target_logits, draft_logits, node_tokens, node_parent, n_pe
                               _ptr(n_per_seq), B, n_uniform, D, _ptr(temperature), per_seq, _ptr(uniforms),
                               _ptr(accepted_len), _ptr(emitted_tokens), _ptr(accepted_nodes), _ptr(row_status),
                               _ptr(diag_p_tok), _ptr(diag_q_tok), _ptr(workspace),
-                              workspace.numel() * workspace.element_size(), ctypes.c_void_p(stream))
+                              workspace.numel() * workspace.element_size(), ctypes.c_void_p(stream),
+                              _path_flags(flags))
     _check(rc)
     return accepted_len, emitted_tokens

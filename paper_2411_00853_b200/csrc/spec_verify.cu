@@ -32,8 +32,6 @@ struct DeviceInfo {
     int ring_argmax_ready[3] = {0, 0, 0};
     int tree_ready[3] = {0, 0, 0};
 };
-std::atomic<int> g_early_exit{0};
-std::atomic<int> g_path{0};   // 0 automatic, 1 streaming kernels, 2 ring kernels where the shape allows
 DeviceInfo g_dev[kMaxDevices];
 std::mutex g_dev_mutex;   // guards the lazy per-device set-up (first call on a device from any thread)
 
@@ -156,11 +154,10 @@ bool ensure_stream_ready(DeviceInfo& dev) {
 template <int DT>
 int launch_ring_path(const specv::BatchView& in, const Workspace& lay, const RingLayout& rl, char* ws,
                      DeviceInfo& dev, int32_t* accepted_len, int32_t* emitted, int32_t* row_status,
-                     float* diag_p, float* diag_q, cudaStream_t stream) {
+                     float* diag_p, float* diag_q, bool early, specv::NextLookahead next, cudaStream_t stream) {
     using namespace specv;
     const size_t smem_stats = sizeof(RingStatsShared), smem_resolve = sizeof(RingResolveShared);
     const size_t smem_early = sizeof(RingEarlyShared);
-    const bool early = g_early_exit.load(std::memory_order_relaxed) != 0;
     if (!ensure_ring_ready<DT>(dev)) return SPECV_ERR_CUDA;
     RingScratch sc;
     sc.off_d = reinterpret_cast<int32_t*>(ws + lay.off_d);
@@ -229,7 +226,7 @@ int launch_ring_path(const specv::BatchView& in, const Workspace& lay, const Rin
     cfg.blockDim = dim3(kRingResolveThreads, 1, 1);
     cfg.dynamicSmemBytes = smem_resolve;
     if (!cuda_ok(cudaLaunchKernelEx(&cfg, specv_ring_resolve<DT>, in, sc, accepted_len, emitted, row_status, diag_p,
-                                    diag_q)))
+                                    diag_q, next)))
         return SPECV_ERR_CUDA;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     trace(3);
@@ -239,7 +236,7 @@ int launch_ring_path(const specv::BatchView& in, const Workspace& lay, const Rin
 template <int DT>
 int launch_stream_path(const specv::BatchView& in, const Workspace& lay, char* ws, DeviceInfo& dev,
                        int32_t* accepted_len, int32_t* emitted, int32_t* row_status,
-                       float* diag_p, float* diag_q, cudaStream_t stream) {
+                       float* diag_p, float* diag_q, specv::NextLookahead next, cudaStream_t stream) {
     using namespace specv;
     int32_t* off_d = reinterpret_cast<int32_t*>(ws + lay.off_d);
     int32_t* seq_status = reinterpret_cast<int32_t*>(ws + lay.seq_status);
@@ -289,7 +286,7 @@ int launch_stream_path(const specv::BatchView& in, const Workspace& lay, char* w
     const int32_t* seq_status_c = seq_status;
     const float2* partial_c = partial;
     if (!cuda_ok(cudaLaunchKernelEx(&cfg, specv_resolve<DT>, in, off_d_c, seq_status_c, partial_c, splits, n_target,
-                                    accepted_len, emitted, row_status, diag_p, diag_q)))
+                                    accepted_len, emitted, row_status, diag_p, diag_q, next)))
         return SPECV_ERR_CUDA;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     trace(3);
@@ -344,6 +341,7 @@ const char* spec_verify_strerror(int status) {
         case SPECV_ERR_ARCH: return "the current device is not compute capability 10.x";
         case SPECV_ERR_TOO_LARGE:
             return "the batch needs more scratch than the built-in buffer of spec_verify_noalloc holds";
+        case SPECV_ERR_FLAGS: return "unknown flag bits, both kernel-set flags, or a flag this call does not take";
         default: return "unknown status";
     }
 }
@@ -375,38 +373,40 @@ int spec_verify_next_lookahead(const int32_t* k_per_row, int32_t k_uniform, cons
 
 int spec_verify_last_path(void) { return g_last_path; }
 
-int spec_verify_set_early_exit(int enable) {
-    g_early_exit.store(enable ? 1 : 0, std::memory_order_relaxed);
-    return SPECV_OK;
+}  // extern "C"
+
+namespace {
+
+constexpr uint32_t kKnownFlags = SPECV_FLAG_STREAMING | SPECV_FLAG_RING | SPECV_FLAG_EARLY_EXIT;
+bool flags_ok(uint32_t flags) {
+    return !(flags & ~kKnownFlags) && (flags & (SPECV_FLAG_STREAMING | SPECV_FLAG_RING)) != (SPECV_FLAG_STREAMING | SPECV_FLAG_RING);
+}
+// Kernel set for a batch of n_items work items whose shape the ring kernels can (or cannot) take.
+// They give a whole (target row, draft row) item to one CTA, so they need enough items to occupy
+// the machine; tiny batches are better served by the streaming kernels, which split rows over CTAs.
+bool choose_ring(uint32_t flags, bool shape_allows, int64_t n_items) {
+    if (!shape_allows || (flags & SPECV_FLAG_STREAMING)) return false;
+    return (flags & SPECV_FLAG_RING) || n_items >= 64;
 }
 
-int spec_verify_set_path(int path) {
-    if (path < 0 || path > 2) return SPECV_ERR_SHAPE;
-    g_path.store(path, std::memory_order_relaxed);
-    return SPECV_OK;
-}
-
-int spec_verify(const void* target_logits, const void* draft_logits, int dtype, int64_t V, int64_t ld_target,
-                int64_t ld_draft, const int32_t* draft_tokens, const int32_t* k_per_row, int32_t B,
-                int32_t k_uniform, int64_t n_draft_total, const float* temperature, int temperature_per_row,
-                const float* uniforms, int32_t* accepted_len, int32_t* emitted_tokens, int32_t* row_status,
-                float* diag_p_tok, float* diag_q_tok, void* workspace, size_t workspace_bytes,
-                void* cuda_stream) {
-    int rc = validate(target_logits, draft_logits, dtype, V, ld_target, ld_draft, draft_tokens, k_per_row, B,
-                      k_uniform, n_draft_total, temperature, uniforms, accepted_len, emitted_tokens);
-    if (rc != SPECV_OK) return rc;
-    if (!workspace) return SPECV_ERR_NULL;
+// Everything after the entry point's own checks of its scratch: the remaining argument checks, the
+// kernel-set choice and the launches.  `ws` holds at least ring_layout(...).total bytes.
+int run_pass(const void* target_logits, const void* draft_logits, int dtype, int64_t V, int64_t ld_target,
+             int64_t ld_draft, const int32_t* draft_tokens, const int32_t* k_per_row, int32_t B, int32_t k_uniform,
+             int64_t n_draft_total, const float* temperature, int temperature_per_row, const float* uniforms,
+             int32_t* accepted_len, int32_t* emitted_tokens, int32_t* row_status, float* diag_p_tok,
+             float* diag_q_tok, char* ws, uint32_t flags, int32_t k_min, int32_t k_max, int32_t* next_k,
+             cudaStream_t stream) {
     const size_t elt = dtype == SPECV_F32 ? 4 : 2;
-    if (!aligned_to(workspace, 256) || !aligned_to(target_logits, elt) || !aligned_to(draft_logits, elt) ||
-        !aligned_to(draft_tokens, 4) || !aligned_to(k_per_row, 4) || !aligned_to(temperature, 4) ||
-        !aligned_to(uniforms, 4) || !aligned_to(accepted_len, 4) || !aligned_to(emitted_tokens, 4) ||
-        !aligned_to(row_status, 4) || !aligned_to(diag_p_tok, 4) || !aligned_to(diag_q_tok, 4))
+    if (!aligned_to(target_logits, elt) || !aligned_to(draft_logits, elt) || !aligned_to(draft_tokens, 4) ||
+        !aligned_to(k_per_row, 4) || !aligned_to(temperature, 4) || !aligned_to(uniforms, 4) ||
+        !aligned_to(accepted_len, 4) || !aligned_to(emitted_tokens, 4) || !aligned_to(row_status, 4) ||
+        !aligned_to(diag_p_tok, 4) || !aligned_to(diag_q_tok, 4) || !aligned_to(next_k, 4))
         return SPECV_ERR_ALIGN;
     const Workspace lay = workspace_layout(B, n_draft_total, V);
     const RingLayout rl = ring_layout(lay.total, B, n_draft_total, V);
-    if (workspace_bytes < rl.total) return SPECV_ERR_WORKSPACE;
     DeviceInfo* dev = nullptr;
-    rc = device_info(&dev);
+    int rc = device_info(&dev);
     if (rc != SPECV_OK) return rc;
 
     specv::BatchView in;
@@ -423,35 +423,66 @@ int spec_verify(const void* target_logits, const void* draft_logits, int dtype, 
     in.temperature = temperature;
     in.per_row_temperature = temperature_per_row ? 1 : 0;
     in.uniforms = uniforms;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    char* ws = static_cast<char*>(workspace);
+    const specv::NextLookahead next{next_k, k_min, k_max};
+    const bool early = (flags & SPECV_FLAG_EARLY_EXIT) != 0;
 
-    // Path choice.  The ring kernels give a whole (target row, draft row) item to one CTA, so
-    // they need enough items to occupy the machine; tiny batches are better served by the
-    // streaming kernels, which split rows over CTAs.
-    const int path = g_path.load(std::memory_order_relaxed);
-    const int64_t n_items = n_draft_total + B;
-    const bool want_ring = ring_shape_ok(in, dtype) && (path == 2 || (path == 0 && n_items >= 64));
-    if (want_ring) {
+    if (choose_ring(flags, ring_shape_ok(in, dtype), n_draft_total + B)) {
         g_last_path = 2;
         if (dtype == SPECV_F32)
             return launch_ring_path<specv::kF32>(in, lay, rl, ws, *dev, accepted_len, emitted_tokens, row_status,
-                                                 diag_p_tok, diag_q_tok, stream);
+                                                 diag_p_tok, diag_q_tok, early, next, stream);
         if (dtype == SPECV_F16)
             return launch_ring_path<specv::kF16>(in, lay, rl, ws, *dev, accepted_len, emitted_tokens, row_status,
-                                                 diag_p_tok, diag_q_tok, stream);
+                                                 diag_p_tok, diag_q_tok, early, next, stream);
         return launch_ring_path<specv::kBF16>(in, lay, rl, ws, *dev, accepted_len, emitted_tokens, row_status,
-                                              diag_p_tok, diag_q_tok, stream);
+                                              diag_p_tok, diag_q_tok, early, next, stream);
     }
     g_last_path = 1;
     if (dtype == SPECV_F32)
         return launch_stream_path<specv::kF32>(in, lay, ws, *dev, accepted_len, emitted_tokens, row_status,
-                                               diag_p_tok, diag_q_tok, stream);
+                                               diag_p_tok, diag_q_tok, next, stream);
     if (dtype == SPECV_F16)
         return launch_stream_path<specv::kF16>(in, lay, ws, *dev, accepted_len, emitted_tokens, row_status,
-                                               diag_p_tok, diag_q_tok, stream);
+                                               diag_p_tok, diag_q_tok, next, stream);
     return launch_stream_path<specv::kBF16>(in, lay, ws, *dev, accepted_len, emitted_tokens, row_status,
-                                            diag_p_tok, diag_q_tok, stream);
+                                            diag_p_tok, diag_q_tok, next, stream);
+}
+
+}  // namespace
+
+extern "C" {
+
+int spec_verify_ex(const void* target_logits, const void* draft_logits, int dtype, int64_t V, int64_t ld_target,
+                   int64_t ld_draft, const int32_t* draft_tokens, const int32_t* k_per_row, int32_t B,
+                   int32_t k_uniform, int64_t n_draft_total, const float* temperature, int temperature_per_row,
+                   const float* uniforms, int32_t* accepted_len, int32_t* emitted_tokens, int32_t* row_status,
+                   float* diag_p_tok, float* diag_q_tok, void* workspace, size_t workspace_bytes,
+                   void* cuda_stream, uint32_t flags, int32_t k_min, int32_t k_max, int32_t* next_k) {
+    int rc = validate(target_logits, draft_logits, dtype, V, ld_target, ld_draft, draft_tokens, k_per_row, B,
+                      k_uniform, n_draft_total, temperature, uniforms, accepted_len, emitted_tokens);
+    if (rc != SPECV_OK) return rc;
+    if (!flags_ok(flags)) return SPECV_ERR_FLAGS;
+    if (next_k && (k_min < 0 || k_max < k_min)) return SPECV_ERR_SHAPE;
+    if (!workspace) return SPECV_ERR_NULL;
+    if (!aligned_to(workspace, 256)) return SPECV_ERR_ALIGN;
+    if (workspace_bytes < ring_layout(workspace_layout(B, n_draft_total, V).total, B, n_draft_total, V).total)
+        return SPECV_ERR_WORKSPACE;
+    return run_pass(target_logits, draft_logits, dtype, V, ld_target, ld_draft, draft_tokens, k_per_row, B, k_uniform,
+                    n_draft_total, temperature, temperature_per_row, uniforms, accepted_len, emitted_tokens,
+                    row_status, diag_p_tok, diag_q_tok, static_cast<char*>(workspace), flags, k_min, k_max, next_k,
+                    static_cast<cudaStream_t>(cuda_stream));
+}
+
+int spec_verify(const void* target_logits, const void* draft_logits, int dtype, int64_t V, int64_t ld_target,
+                int64_t ld_draft, const int32_t* draft_tokens, const int32_t* k_per_row, int32_t B,
+                int32_t k_uniform, int64_t n_draft_total, const float* temperature, int temperature_per_row,
+                const float* uniforms, int32_t* accepted_len, int32_t* emitted_tokens, int32_t* row_status,
+                float* diag_p_tok, float* diag_q_tok, void* workspace, size_t workspace_bytes,
+                void* cuda_stream) {
+    return spec_verify_ex(target_logits, draft_logits, dtype, V, ld_target, ld_draft, draft_tokens, k_per_row, B,
+                          k_uniform, n_draft_total, temperature, temperature_per_row, uniforms, accepted_len,
+                          emitted_tokens, row_status, diag_p_tok, diag_q_tok, workspace, workspace_bytes, cuda_stream,
+                          0u, 0, 0, nullptr);
 }
 
 namespace {
@@ -672,10 +703,11 @@ extern "C" int spec_verify_tree(const void* target_logits, const void* draft_log
                                 int temperature_per_seq, const float* uniforms, int32_t* accepted_len,
                                 int32_t* emitted_tokens, int32_t* accepted_nodes, int32_t* row_status,
                                 float* diag_p_tok, float* diag_q_tok, void* workspace, size_t workspace_bytes,
-                                void* cuda_stream) {
+                                void* cuda_stream, uint32_t flags) {
     int rc = validate(target_logits, draft_logits, dtype, V, ld_target, ld_draft, node_tokens, n_per_seq, B,
                       n_uniform, n_node_total, temperature, uniforms, accepted_len, emitted_tokens);
     if (rc != SPECV_OK) return rc;
+    if (!flags_ok(flags) || (flags & SPECV_FLAG_EARLY_EXIT)) return SPECV_ERR_FLAGS;
     if (!workspace || (n_node_total > 0 && !node_parent)) return SPECV_ERR_NULL;
     const size_t elt = dtype == SPECV_F32 ? 4 : 2;
     if (!aligned_to(workspace, 256) || !aligned_to(target_logits, elt) || !aligned_to(draft_logits, elt) ||
@@ -705,8 +737,7 @@ extern "C" int spec_verify_tree(const void* target_logits, const void* draft_log
     in.per_row_temperature = temperature_per_seq ? 1 : 0;
     in.uniforms = uniforms;
     in.parent = node_parent;
-    const int path = g_path.load(std::memory_order_relaxed);
-    const bool ring = ring_shape_ok(in, dtype) && (path == 2 || (path == 0 && n_node_total + B >= 64));
+    const bool ring = choose_ring(flags, ring_shape_ok(in, dtype), n_node_total + B);
     g_last_path = ring ? 2 : 1;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
@@ -827,8 +858,9 @@ extern "C" int spec_verify_greedy(const void* target_logits, int dtype, int64_t 
                                   const int32_t* draft_tokens, const int32_t* k_per_row, int32_t B,
                                   int32_t k_uniform, int64_t n_draft_total, int32_t* accepted_len,
                                   int32_t* emitted_tokens, int32_t* row_status, int32_t* target_argmax,
-                                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream, uint32_t flags) {
     if (dtype != SPECV_F32 && dtype != SPECV_BF16 && dtype != SPECV_F16) return SPECV_ERR_DTYPE;
+    if (!flags_ok(flags) || (flags & SPECV_FLAG_EARLY_EXIT)) return SPECV_ERR_FLAGS;
     if (!shape_ok(B, n_draft_total, V) || ld_target < V) return SPECV_ERR_SHAPE;
     if (!k_per_row && (k_uniform < 0 || (int64_t)B * k_uniform != n_draft_total)) return SPECV_ERR_SHAPE;
     if (!target_logits || !accepted_len || !emitted_tokens || !workspace) return SPECV_ERR_NULL;
@@ -859,9 +891,8 @@ extern "C" int spec_verify_greedy(const void* target_logits, int dtype, int64_t 
     in.per_row_temperature = 0;
     in.uniforms = nullptr;
     // the ring kernel gives a whole row to one CTA: it needs enough rows to occupy the machine
-    const int path = g_path.load(std::memory_order_relaxed);
     const bool bulk_ok = !(reinterpret_cast<uintptr_t>(in.target) & 15u) && !(in.pitch_t & 15) && !((V * (int64_t)elt) & 15);
-    const bool ring = bulk_ok && (path == 2 || (path == 0 && n_draft_total + B >= 64));
+    const bool ring = choose_ring(flags, bulk_ok, n_draft_total + B);
     g_last_path = ring ? 2 : 1;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     char* ws = static_cast<char*>(workspace);
@@ -876,7 +907,7 @@ extern "C" int spec_verify_greedy(const void* target_logits, int dtype, int64_t 
 }
 
 // ---------------------------------------------------------------------------------
-// spec_verify_noalloc: the streaming kernel set with its scratch in a static device array.
+// spec_verify_noalloc: spec_verify with its scratch in a static device array.
 // ---------------------------------------------------------------------------------
 namespace {
 
@@ -914,45 +945,16 @@ extern "C" int spec_verify_noalloc(const void* target_logits, const void* draft_
     int rc = validate(target_logits, draft_logits, dtype, V, ld_target, ld_draft, draft_tokens, k_per_row, B,
                       k_uniform, n_draft_total, temperature, uniforms, accepted_len, emitted_tokens);
     if (rc != SPECV_OK) return rc;
-    const Workspace lay = workspace_layout(B, n_draft_total, V);
-    if (ring_layout(lay.total, B, n_draft_total, V).total > (size_t)SPECV_NOALLOC_SCRATCH_BYTES)
+    if (ring_layout(workspace_layout(B, n_draft_total, V).total, B, n_draft_total, V).total >
+        (size_t)SPECV_NOALLOC_SCRATCH_BYTES)
         return SPECV_ERR_TOO_LARGE;   // the documented limit is the public workspace size
-    const size_t elt = dtype == SPECV_F32 ? 4 : 2;
-    if (!aligned_to(target_logits, elt) || !aligned_to(draft_logits, elt) || !aligned_to(draft_tokens, 4) ||
-        !aligned_to(k_per_row, 4) || !aligned_to(temperature, 4) || !aligned_to(uniforms, 4) ||
-        !aligned_to(accepted_len, 4) || !aligned_to(emitted_tokens, 4) || !aligned_to(row_status, 4) ||
-        !aligned_to(diag_p_tok, 4) || !aligned_to(diag_q_tok, 4))
-        return SPECV_ERR_ALIGN;
-    DeviceInfo* dev = nullptr;
-    rc = device_info(&dev);
-    if (rc != SPECV_OK) return rc;
     char* scratch = nullptr;
     rc = static_scratch_for_current_device(&scratch);
     if (rc != SPECV_OK) return rc;
-
-    specv::BatchView in;
-    in.target = static_cast<const char*>(target_logits);
-    in.draft = static_cast<const char*>(draft_logits);
-    in.pitch_t = ld_target * (int64_t)elt;
-    in.pitch_d = ld_draft * (int64_t)elt;
-    in.V = V;
-    in.tokens = draft_tokens;
-    in.k_per_row = k_per_row;
-    in.B = B;
-    in.k_uniform = k_uniform;
-    in.n_draft_total = n_draft_total;
-    in.temperature = temperature;
-    in.per_row_temperature = temperature_per_row ? 1 : 0;
-    in.uniforms = uniforms;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    // Nothing in the scratch has to start at zero: the prologue kernel writes the offsets and
-    // the per-sequence status, the statistics kernel writes every partial, before any is read.
-    if (dtype == SPECV_F32)
-        return launch_stream_path<specv::kF32>(in, lay, scratch, *dev, accepted_len, emitted_tokens, row_status,
-                                               diag_p_tok, diag_q_tok, stream);
-    if (dtype == SPECV_F16)
-        return launch_stream_path<specv::kF16>(in, lay, scratch, *dev, accepted_len, emitted_tokens, row_status,
-                                               diag_p_tok, diag_q_tok, stream);
-    return launch_stream_path<specv::kBF16>(in, lay, scratch, *dev, accepted_len, emitted_tokens, row_status,
-                                            diag_p_tok, diag_q_tok, stream);
+    // Nothing in the scratch has to start at zero: whichever kernel set runs writes every word of
+    // it (offsets, per-sequence status, statistics, tickets) before reading it.
+    return run_pass(target_logits, draft_logits, dtype, V, ld_target, ld_draft, draft_tokens, k_per_row, B, k_uniform,
+                    n_draft_total, temperature, temperature_per_row, uniforms, accepted_len, emitted_tokens,
+                    row_status, diag_p_tok, diag_q_tok, scratch, 0u, 0, 0, nullptr,
+                    static_cast<cudaStream_t>(cuda_stream));
 }

@@ -862,7 +862,7 @@ __device__ __forceinline__ void consume_resolve_unit(ChunkRing& ring, RingRun& r
 template <int DT>
 __device__ __forceinline__ void locate_and_emit(const BatchView& in, const SeqRecord& r, float* seg, int32_t nseg,
                                                 int32_t* result_slot, int lane, int32_t* accepted_len,
-                                                int32_t* emitted, int32_t* row_status) {
+                                                int32_t* emitted, int32_t* row_status, const NextLookahead& next) {
     auto wsync = [] { __syncwarp(); };
     int status = r.status;
     SampleRows sr = r.rows;
@@ -880,6 +880,8 @@ __device__ __forceinline__ void locate_and_emit(const BatchView& in, const SeqRe
     if (lane == 0) {
         accepted_len[r.b] = r.n;
         if (row_status) row_status[r.b] = status;
+        // a sequence that draws a token is valid, so r.K is its lookahead as the caller gave it
+        if (next.out) next.out[r.b] = next_lookahead_of(r.K, r.n, next.k_min, next.k_max);
     }
 }
 
@@ -917,7 +919,8 @@ static_assert(kPartDepth == kCWarps, "the first kPartDepth records are produced 
 template <int DT>
 __global__ void __launch_bounds__(kRingResolveThreads, 1)
 specv_ring_resolve(BatchView in, RingScratch ws, int32_t* __restrict__ accepted_len, int32_t* __restrict__ emitted,
-                   int32_t* __restrict__ row_status, float* __restrict__ diag_p, float* __restrict__ diag_q) {
+                   int32_t* __restrict__ row_status, float* __restrict__ diag_p, float* __restrict__ diag_q,
+                   NextLookahead next) {
     using E = Elt<DT>;
     constexpr int SEG = 32 * E::kPerVec;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -978,6 +981,9 @@ specv_ring_resolve(BatchView in, RingScratch ws, int32_t* __restrict__ accepted_
                 if (lane == 0) {
                     accepted_len[b] = 0;
                     if (row_status) row_status[b] = r.stream ? 16 : r.status;   // 16: SPECV_ROW_INTERNAL
+                    if (next.out)
+                        next.out[b] = next_lookahead_of(in.k_per_row ? in.k_per_row[b] : in.k_uniform, 0, next.k_min,
+                                                        next.k_max);
                 }
             }
             if (lane == 0) {
@@ -1084,7 +1090,7 @@ specv_ring_resolve(BatchView in, RingScratch ws, int32_t* __restrict__ accepted_
                 const float* gs = ws.gseg + (int64_t)r.b * nseg;
                 for (int32_t i = lane; i < nseg; i += 32) sh.seg[i] = __ldcg(gs + i);
                 __syncwarp();
-                locate_and_emit<DT>(in, r, sh.seg, nseg, &sh.result_slot, lane, accepted_len, emitted, row_status);
+                locate_and_emit<DT>(in, r, sh.seg, nseg, &sh.result_slot, lane, accepted_len, emitted, row_status, next);
                 __syncwarp();
             }
         }

@@ -34,6 +34,18 @@ struct BatchView {
     const int32_t* ctx_has_children = nullptr;
 };
 
+// Lookahead of the next speculation round, written by the kernel that emits a sequence's tokens
+// (out == nullptr: not wanted): K+2 after a fully accepted draft, else K-1, within [k_min, k_max].
+struct NextLookahead {
+    int32_t* out;
+    int32_t k_min, k_max;
+};
+__device__ __forceinline__ int32_t next_lookahead_of(int32_t k_raw, int32_t accepted, int32_t k_min, int32_t k_max) {
+    const int32_t K = k_raw > 0 ? k_raw : 0;
+    const int32_t next = accepted >= K ? K + 2 : K - 1;
+    return min(max(next, k_min), k_max);
+}
+
 // ---------------------------------------------------------------------------------
 // Prologue.  Block 0 scans max(K_b,0) into off_d[0..B] and records per-sequence
 // argument errors; all blocks fill emitted_tokens with -1.
@@ -437,7 +449,8 @@ __global__ void __launch_bounds__(kResolveThreads)
 specv_resolve(BatchView in, const int32_t* __restrict__ off_d, const int32_t* __restrict__ seq_status,
               const float2* __restrict__ partial, int splits, int64_t n_target_rows,
               int32_t* __restrict__ accepted_len, int32_t* __restrict__ emitted,
-              int32_t* __restrict__ row_status, float* __restrict__ diag_p, float* __restrict__ diag_q) {
+              int32_t* __restrict__ row_status, float* __restrict__ diag_p, float* __restrict__ diag_q,
+              NextLookahead next) {
     using E = Elt<DT>;
     extern __shared__ float seg[];
     __shared__ int32_t first_reject;
@@ -468,6 +481,7 @@ specv_resolve(BatchView in, const int32_t* __restrict__ off_d, const int32_t* __
         if (tid == 0) {
             accepted_len[b] = 0;
             if (row_status) row_status[b] = status;
+            if (next.out) next.out[b] = next_lookahead_of(k_raw, 0, next.k_min, next.k_max);
         }
         return;   // the prologue already wrote -1 into every slot
     }
@@ -535,6 +549,7 @@ specv_resolve(BatchView in, const int32_t* __restrict__ off_d, const int32_t* __
     if (tid == 0) {
         accepted_len[b] = n;
         if (row_status) row_status[b] = status;
+        if (next.out) next.out[b] = next_lookahead_of(k_raw, n, next.k_min, next.k_max);
     }
 }
 
@@ -546,10 +561,7 @@ __global__ void specv_next_lookahead(const int32_t* __restrict__ k_per_row, int3
                                      int32_t k_max, int32_t* __restrict__ next_k) {
     const int32_t b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
-    int32_t K = k_per_row ? k_per_row[b] : k_uniform;
-    if (K < 0) K = 0;
-    int32_t next = accepted_len[b] >= K ? K + 2 : K - 1;
-    next_k[b] = min(max(next, k_min), k_max);
+    next_k[b] = next_lookahead_of(k_per_row ? k_per_row[b] : k_uniform, accepted_len[b], k_min, k_max);
 }
 
 }  // namespace specv

@@ -68,7 +68,7 @@ def read_hand_cases():
                 continue
             key, _, rest = line.partition(" ")
             if key == "case":
-                cur = {"name": rest.strip(), "zero_margin": False}
+                cur = {"name": rest.strip(), "zero_margin": False, "no_crossing": False}
                 cases.append(cur)
             elif key in ("target", "draft"):
                 rows = [r.split() for r in rest.split(";")] if rest.strip() else []
@@ -77,7 +77,7 @@ def read_hand_cases():
                 cur["T"] = float(rest)
             elif key == "tokens":
                 cur["tokens"] = [int(v) for v in rest.split()]
-            elif key in ("u", "expect_ptok", "expect_qtok"):
+            elif key in ("u", "expect_ptok", "expect_qtok", "expect_rho"):
                 cur[key] = [float(v) for v in rest.split()]
             elif key == "expect_len":
                 cur["expect_len"] = int(rest)
@@ -85,6 +85,8 @@ def read_hand_cases():
                 cur["expect_emitted"] = [int(v) for v in rest.split()]
             elif key == "zero_margin":
                 cur["zero_margin"] = True
+            elif key == "no_crossing":
+                cur["no_crossing"] = True
             else:
                 raise ValueError(f"unknown key {key!r} in hand_cases.txt")
     return cases
@@ -131,3 +133,47 @@ def classify_rows(ora, k_per_row, got_len, got_emitted, off_d, off_t, margin=MAR
         else:
             failures.append(b)
     return identical, excused, failures
+
+
+class Case:
+    """Packed numpy arrays with the Workload fields the test helpers use."""
+    def __init__(self, tl, dl, tok, k, T, uni, dtype="f32"):
+        self.target_logits, self.draft_logits, self.draft_tokens = tl, dl, tok
+        self.k_per_row, self.temperature, self.uniforms = k, T, uni
+        self.B, self.V, self.dtype = len(k), tl.shape[1], dtype
+        self.off_d = np.concatenate([[0], np.cumsum(k)]).astype(np.int64)
+        self.off_t = self.off_d[:-1] + np.arange(self.B)
+        self.n_draft_total = int(self.off_d[-1])
+
+
+def neg_inf_of(a: np.ndarray):
+    """-inf in the storage type of a logits array (bf16 is stored as uint16 bit patterns)."""
+    return np.uint16(0xFF80) if a.dtype == np.uint16 else a.dtype.type(-np.inf)
+
+
+def masked_case(w, seed: int, contiguous_every: int = 3):
+    """Workload w with half of every sequence's vocabulary masked by -inf logits, the way a
+    constrained sampler masks forbidden tokens: per sequence one set of kept ids (exactly
+    V // 2 of them), applied to all its target and draft rows; every `contiguous_every`-th
+    sequence keeps the SECOND half of the vocabulary instead of a random half, so that whole
+    vectors, lanes and chunks of a row hold nothing but -inf.  Drafted tokens are moved onto
+    kept ids.  Returns (case, kept) with kept[b] the sorted kept ids of sequence b."""
+    rng = np.random.default_rng(seed)
+    tl, dl, tok = w.target_logits.copy(), w.draft_logits.copy(), w.draft_tokens.copy()
+    ninf = neg_inf_of(tl)
+    V, kept = w.V, []
+    for b in range(w.B):
+        if b % contiguous_every == contiguous_every - 1:
+            keep = np.arange(V - V // 2, V)
+        else:
+            keep = np.sort(rng.choice(V, V // 2, replace=False))
+        kept.append(keep)
+        gone = np.ones(V, bool)
+        gone[keep] = False
+        K = int(w.k_per_row[b])
+        tl[w.off_t[b]:w.off_t[b] + K + 1, gone] = ninf
+        dl[w.off_d[b]:w.off_d[b] + K, gone] = ninf
+        for i in range(K):
+            x = tok[w.off_d[b] + i]
+            tok[w.off_d[b] + i] = keep[np.searchsorted(keep, x) % len(keep)]
+    return Case(tl, dl, tok, w.k_per_row, w.temperature, w.uniforms, dtype=w.dtype), kept

@@ -10,30 +10,23 @@ import torch
 
 import oracle
 from gpu_utils import DeviceBatch, assert_parity, run_oracle
-from helpers import hand_case_inputs, read_hand_cases
+from helpers import Case, hand_case_inputs, read_hand_cases
 from paper_2411_00853_b200 import binding
 from paper_2411_00853_b200 import workloads as W
 
 pytestmark = [pytest.mark.gpu, pytest.mark.usefixtures("kernel_path")]
 
 
-class _Case:
-    """Adapter: packed numpy arrays -> the Workload fields the helpers use."""
-    def __init__(self, tl, dl, tok, k, T, uni, dtype="f32"):
-        self.target_logits, self.draft_logits, self.draft_tokens = tl, dl, tok
-        self.k_per_row, self.temperature, self.uniforms = k, T, uni
-        self.B, self.V, self.dtype = len(k), tl.shape[1], dtype
-        self.off_d = np.concatenate([[0], np.cumsum(k)]).astype(np.int64)
-        self.off_t = self.off_d[:-1] + np.arange(self.B)
-        self.n_draft_total = int(self.off_d[-1])
+_Case = Case
 
 
 @pytest.mark.parametrize("case", [c for c in read_hand_cases() if not c["zero_margin"]],
                          ids=lambda c: c["name"])
-def test_hand_cases(case):
+def test_hand_cases(kernel_path, case):
     w = _Case(*hand_case_inputs(case))
     acc, em, st, dp, dq = DeviceBatch(w).run()
     assert acc[0] == case["expect_len"] and em.tolist() == case["expect_emitted"] and st[0] == 0
+    assert binding.last_path() == (binding.PATH_RING if kernel_path == "ring" else binding.PATH_STREAMING)
     if "expect_ptok" in case:
         np.testing.assert_allclose(dp, case["expect_ptok"], rtol=1e-5)
         np.testing.assert_allclose(dq, case["expect_qtok"], rtol=1e-5)
@@ -171,6 +164,21 @@ def test_argument_errors_come_back_as_status_codes():
     assert call(dtype=3) == 3
     assert call(ws=dev.workspace.data_ptr() + 4) == 4 and call(tok=dev.tokens.data_ptr() + 2) == 4
     assert call(wsb=16) == 5
+
+    def call_ex(flags, k_min=0, k_max=0, next_k=None):
+        return lib.spec_verify_ex(dev.target.data_ptr(), dev.draft.data_ptr(), 1, 512, 512, 512,
+                                  dev.tokens.data_ptr(), dev.k.data_ptr(), 2, 0, 10, dev.temperature.data_ptr(), 0,
+                                  dev.uniforms.data_ptr(), dev.accepted.data_ptr(), dev.emitted.data_ptr(), None,
+                                  None, None, dev.workspace.data_ptr(), dev.workspace.numel(), None, flags, k_min,
+                                  k_max, next_k)
+
+    assert call_ex(0) == 0 and call_ex(binding.FLAG_RING | binding.FLAG_EARLY_EXIT) == 0
+    assert call_ex(binding.FLAG_RING | binding.FLAG_STREAMING) == 9 and call_ex(8) == 9 and call_ex(1 << 31) == 9
+    nk = torch.zeros(2, dtype=torch.int32, device="cuda")
+    assert call_ex(0, 1, 8, nk.data_ptr()) == 0
+    assert call_ex(0, -1, 8, nk.data_ptr()) == 2 and call_ex(0, 5, 4, nk.data_ptr()) == 2
+    assert call_ex(0, 5, 4, None) == 0                    # the bounds only matter with next_k
+    assert call_ex(0, 1, 8, nk.data_ptr() + 2) == 4
     torch.cuda.synchronize()
 
 

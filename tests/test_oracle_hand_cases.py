@@ -15,8 +15,9 @@ CASES = read_hand_cases()
 
 
 def test_fixture_is_complete():
-    assert len(CASES) >= 12
-    assert {c["name"][:2] for c in CASES} >= {"H1", "H2", "H3", "H4", "H5", "H6", "H7", "H8"}
+    assert len(CASES) >= 16
+    assert {c["name"].split("_")[0].rstrip("ab") for c in CASES} >= {"H1", "H2", "H3", "H4", "H5", "H6", "H7", "H8",
+                                                                       "H9", "H10"}
 
 
 @pytest.mark.parametrize("case", CASES, ids=[c["name"] for c in CASES])
@@ -32,13 +33,18 @@ def test_hand_case(case):
         return
     assert res.accepted_len[0] == case["expect_len"]
     assert res.emitted_tokens.tolist() == case["expect_emitted"]
-    if case["u"][-1] > 0:   # u' = 0 touches the (empty) step below the first massive token
+    if case["no_crossing"]:
+        # u' = 1: the threshold is the whole mass, so the draw is decided by the "largest id with
+        # mass" convention (or by a last cumulative value that rounding put above the total)
+        assert res.cdf_margin[0] < 1e-12
+    elif case["u"][-1] > 0:   # u' = 0 touches the (empty) step below the first massive token
         assert res.cdf_margin[0] > 5e-4
     if "expect_ptok" in case:
         np.testing.assert_allclose(res.p_tok, case["expect_ptok"], rtol=1e-6)
         np.testing.assert_allclose(res.q_tok, case["expect_qtok"], rtol=1e-6)
-        np.testing.assert_allclose(res.rho, np.array(case["expect_ptok"]) / np.array(case["expect_qtok"]),
-                                   rtol=1e-6)
+        rho = (case["expect_rho"] if "expect_rho" in case
+               else np.array(case["expect_ptok"]) / np.array(case["expect_qtok"]))
+        np.testing.assert_allclose(res.rho, rho, rtol=1e-6)
 
 
 def test_hand_cases_batched_ragged():

@@ -11,7 +11,7 @@ import pytest
 from scipy.special import logsumexp
 
 import oracle
-from helpers import bf16_bits_to_f64, f32_to_bf16_bits, logits_as_f64, pack
+from helpers import Case, bf16_bits_to_f64, f32_to_bf16_bits, logits_as_f64, masked_case, neg_inf_of, pack
 from paper_2411_00853_b200 import workloads as W
 
 
@@ -236,6 +236,66 @@ def test_one_hot_target_always_emits_the_hot_token():
         assert res.emitted_tokens[off_t[b]] == s["hot"]            # accepted draft or resampled: the hot token
         if res.accepted_len[b] == 1:
             assert res.emitted_tokens[off_t[b] + 1] == s["hot"]    # bonus too
+
+
+# ---------------------------------------------------------------- masked logits (-inf)
+@pytest.mark.parametrize("cfg,V", [(1, 64), (5, 200), (2, 1024)])
+def test_masked_logits_equal_the_compacted_vocabulary(cfg, V):
+    """A logit of -inf is a token of probability 0 under either model, so masking half of the
+    vocabulary must give exactly what the pass gives on the vocabulary with those ids removed:
+    same accepted lengths, same probabilities of the drafted tokens, and emitted tokens that
+    are the compacted run's tokens mapped back to the original ids."""
+    w = W.make_config(cfg, B=18, V=V)
+    m, kept = masked_case(w, seed=cfg)
+    full = run(m)
+    assert np.all(full.row_status == 0)
+    # the compacted batch: every sequence keeps V // 2 ids, so the batch stays rectangular
+    ctl = np.empty((m.target_logits.shape[0], V // 2), m.target_logits.dtype)
+    cdl = np.empty((m.draft_logits.shape[0], V // 2), m.draft_logits.dtype)
+    ctok = m.draft_tokens.copy()
+    for b in range(m.B):
+        K = int(m.k_per_row[b])
+        ctl[m.off_t[b]:m.off_t[b] + K + 1] = m.target_logits[m.off_t[b]:m.off_t[b] + K + 1][:, kept[b]]
+        cdl[m.off_d[b]:m.off_d[b] + K] = m.draft_logits[m.off_d[b]:m.off_d[b] + K][:, kept[b]]
+        ctok[m.off_d[b]:m.off_d[b] + K] = np.searchsorted(kept[b], m.draft_tokens[m.off_d[b]:m.off_d[b] + K])
+    small = oracle.spec_verify(ctl, cdl, ctok, m.k_per_row, m.temperature, m.uniforms)
+    assert np.array_equal(full.accepted_len, small.accepted_len)
+    np.testing.assert_allclose(full.p_tok, small.p_tok, rtol=1e-12)
+    np.testing.assert_allclose(full.q_tok, small.q_tok, rtol=1e-12)
+    checked = 0
+    for b in range(m.B):
+        if min(full.cdf_margin[b], small.cdf_margin[b]) < 1e-12:
+            continue
+        n = int(full.accepted_len[b])
+        assert full.emitted_tokens[m.off_t[b] + n] == kept[b][small.emitted_tokens[m.off_t[b] + n]]
+        assert not np.isneginf(logits_as_f64(m.target_logits[m.off_t[b] + n])[full.emitted_tokens[m.off_t[b] + n]])
+        checked += 1
+    assert checked >= m.B - 2
+
+
+def test_rows_without_any_mass():
+    """Degenerate rows made of -inf only (a mask that forbids everything) have no distribution.
+    Stated behaviour: a drafted token scored by such a row is rejected; a draw from such a row
+    yields the last token id; a residual that cannot be formed falls back to the target row and
+    raises the zero-residual bit."""
+    V, rng = 24, np.random.default_rng(21)
+    ninf = np.float32(-np.inf)
+    def seq(K):
+        tl = rng.normal(0, 2, (K + 1, V)).astype(np.float32)
+        return {"target": tl, "draft": tl[:K].copy(), "tokens": list(rng.integers(0, V, K)),
+                "u": [np.float32(0.5)] * K, "u2": np.float32(0.4)}
+    a, b, c, d = seq(2), seq(2), seq(2), seq(2)
+    a["target"][1] = ninf                 # a: target row of position 1 empty -> rejected there, draw impossible
+    b["target"][2] = ninf                 # b: identical models accept everything, the bonus row is empty
+    c["draft"][0] = ninf                  # c: draft row of position 0 empty -> rejected, resampled from the target row
+    tl, dl, tok, k, uni, off_d, off_t = pack([a, b, c, d], V)
+    res = oracle.spec_verify(tl, dl, tok, k, np.array([1.0], np.float32), uni)
+    assert res.accepted_len.tolist() == [1, 2, 0, 2]
+    assert res.emitted_tokens[off_t[0] + 1] == V - 1 and res.row_status[0] == oracle.ROW_ZERO_RESIDUAL
+    assert res.emitted_tokens[off_t[1] + 2] == V - 1 and res.row_status[1] == 0
+    assert res.row_status[2] == oracle.ROW_ZERO_RESIDUAL
+    assert res.emitted_tokens[off_t[2]] == numpy_sampler(c["target"][0].astype(np.float64), 1.0, 0.4)
+    assert res.row_status[3] == 0
 
 
 # ---------------------------------------------------------------- layout and data errors

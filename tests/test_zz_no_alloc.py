@@ -7,10 +7,12 @@ allocation may bring.  They cannot supply spec_verify's workspace, so the librar
 fixed 4 MiB scratch array in its device image and this entry point uses it.
 
 The array is shared by all calls and keeps the previous call's contents, so the test makes
-two calls in a row on DIFFERENT batches (the second smaller and of another dtype, so stale
-words from the first would sit exactly where the second reads) and requires each to give
-what the ordinary entry point gives on the same inputs: identical lengths, tokens and
-status, probabilities within the 1e-5 relative tolerance of the parity tests.  It is kept
+calls in a row on DIFFERENT batches (of different size, dtype and kernel set, so stale words
+from one would sit exactly where the next reads) and requires each to give what the ordinary
+entry point gives on the same inputs.  Both entry points run the same kernels on the same
+batch (same automatic choice of the kernel set), so lengths, tokens and status are identical
+and the probabilities agree far inside the 1e-5 relative tolerance of the parity tests; the
+results are also held against the fp64 oracle under the usual margin rule.  It is kept
 in a file that sorts last so that a run stopping at the first failure has already run
 every other test; it passes alone in a fresh process as well as after the others.
 """
@@ -20,7 +22,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_utils import PROB_RTOL, DeviceBatch
+from gpu_utils import PROB_RTOL, DeviceBatch, assert_parity
 from paper_2411_00853_b200 import binding
 from paper_2411_00853_b200 import workloads as W
 
@@ -48,13 +50,28 @@ def _same(got, ref):
     np.testing.assert_allclose(got[4], ref[4], rtol=PROB_RTOL, atol=1e-37)
 
 
-def test_two_calls_in_a_row_match_the_workspace_entry_point():
-    first = DeviceBatch(W.make_config(5, B=48, V=20000))      # bf16, ragged lookahead, split rows
-    second = DeviceBatch(W.make_config(1, B=3, V=4099))       # fp32, fewer rows: reuses the dirty scratch
-    ref_first, ref_second = first.run(), second.run()
-    _same(_noalloc(first), ref_first)
-    _same(_noalloc(second), ref_second)
+def test_calls_in_a_row_match_the_workspace_entry_point():
+    binding.set_path(binding.PATH_AUTO)
+    first = DeviceBatch(W.make_config(5, B=48, V=20000))      # bf16, ragged lookahead: ring kernels
+    second = DeviceBatch(W.make_config(1, B=3, V=4099))       # fp32, few odd rows: streaming kernels
+    ref_first = first.run()
+    assert binding.last_path() == binding.PATH_RING
+    ref_second = second.run()
+    assert binding.last_path() == binding.PATH_STREAMING
+    got = _noalloc(first)
+    assert binding.last_path() == binding.PATH_RING           # the same kernel set as spec_verify chose
+    _same(got, ref_first)
+    assert_parity(first.w, got)
+    got = _noalloc(second)                                    # reuses the scratch the ring kernels left dirty
+    assert binding.last_path() == binding.PATH_STREAMING
+    _same(got, ref_second)
+    assert_parity(second.w, got)
     _same(_noalloc(first), ref_first)                          # and back again
+
+
+def test_the_largest_benchmark_shape_fits_the_built_in_scratch():
+    """512 ragged sequences over a vocabulary of 128256 need 2.3 MiB of the 4 MiB."""
+    assert 0 < binding.workspace_bytes(512, 4400, 128256) <= binding.NOALLOC_SCRATCH_BYTES
 
 
 def test_batches_beyond_the_built_in_scratch_are_refused():
