@@ -68,6 +68,8 @@ class ClockSampler(threading.Thread):
         super().__init__(daemon=True)
         self.period = period_s
         self.samples, self.reasons = [], 0
+        self.by_region = {}
+        self.region_name = None
         self.max_mhz = None
         self._stop_evt = threading.Event()
         self._active = threading.Event()
@@ -97,14 +99,30 @@ class ClockSampler(threading.Thread):
                         r = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
                     except Exception:
                         r = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
-                    self.samples.append(mhz)
-                    self.reasons |= r
+                    name = self.region_name
+                    if name == "main":
+                        self.samples.append(mhz)
+                        self.reasons |= r
+                    reg = self.by_region.setdefault(name, [[], 0])
+                    reg[0].append(mhz)
+                    reg[1] |= r
                 except Exception:
                     pass
             time.sleep(self.period)
 
-    def region(self, on: bool):
-        (self._active.set if on else self._active.clear)()
+    def region(self, on: bool, name: str = "main"):
+        """Samples taken while a region is on are filed under its name; "main" is the timed region of
+        the headline figure."""
+        if on:
+            self.region_name = name
+            self._active.set()
+        else:
+            self._active.clear()
+
+    def region_summary(self, name: str):
+        mhz, reasons = self.by_region.get(name, [[], 0])
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(v for k, v in self.REASONS.items() if reasons & k), "samples": len(mhz)}
 
     def stop(self):
         self._stop_evt.set()
@@ -120,8 +138,22 @@ class ClockSampler(threading.Thread):
 def workload_config(w, cfg):
     return {"workload": f"config{cfg}: {w.recipe}", "B": int(w.B), "V": int(w.V), "logits_dtype": w.dtype,
             "draft_positions": int(w.n_draft_total), "logit_bytes": int(w.logit_bytes),
-            "l2": "inputs larger than L2 (every pass streams %.0f MB)" % (w.logit_bytes / 1e6)
-            if w.logit_bytes > 2 * L2_BYTES else "L2 flushed between timed iterations"}
+            "l2": ("L2 flushed between timed iterations (a 252 MB buffer is read)" if needs_flush(w) else
+                   "inputs larger than L2 (every pass streams %.0f MB, %.0f times the L2%s)" % (
+                       w.logit_bytes / 1e6, w.logit_bytes / L2_BYTES,
+                       "; consecutive passes rotate through 3 distinct copies of the logits" if input_sets(w) > 1 else ""))}
+
+
+def needs_flush(w) -> bool:
+    """A workload that fits in L2 is timed with an L2 flush between passes."""
+    return w.logit_bytes <= 2 * L2_BYTES
+
+
+def input_sets(w) -> int:
+    """Distinct copies of the logits that consecutive passes rotate through: three for workloads
+    between 2 and 8 times the L2 (so that no pass can find lines of its own input left by an
+    earlier pass), one otherwise."""
+    return 3 if 2 * L2_BYTES < w.logit_bytes < 8 * L2_BYTES else 1
 
 
 # --------------------------------------------------------------------------- reference arm
@@ -173,22 +205,56 @@ class DeviceWorkload:
                          temperature=torch.from_numpy(np.ascontiguousarray(w.temperature)),
                          uniforms=torch.from_numpy(np.ascontiguousarray(w.uniforms)))
         self.dev = {k: v.to(device) for k, v in self.host.items()}
+        # consecutive passes rotate through these copies of the logits (see input_sets)
+        self.logit_sets = [(self.dev["target"], self.dev["draft"])]
+        for _ in range(input_sets(w) - 1):
+            self.logit_sets.append((self.dev["target"].clone(), self.dev["draft"].clone()))
+        self.calls = 0
         D, B, V = w.n_draft_total, w.B, w.V
         self.accepted = torch.empty(B, dtype=torch.int32, device=device)
         self.emitted = torch.empty(D + B, dtype=torch.int32, device=device)
         self.workspace = torch.empty(max(256, binding.workspace_bytes(B, D, V)), dtype=torch.uint8, device=device)
         self.binding = binding
         self.stream = torch.cuda.current_stream(device).cuda_stream
+        # a batch whose sequences all have the same lookahead is passed the way a caller with a
+        # fixed lookahead would pass it: k_per_row = NULL, k_uniform = K
+        k = np.asarray(w.k_per_row)
+        self.k_uniform = int(k[0]) if k.size and np.all(k == k[0]) else None
 
     def step(self):
         d = self.dev
-        self.binding.spec_verify(d["target"], d["draft"], d["tokens"], d["k"], d["temperature"], d["uniforms"],
+        target, draft = self.logit_sets[self.calls % len(self.logit_sets)]
+        self.calls += 1
+        self.binding.spec_verify(target, draft, d["tokens"], None if self.k_uniform is not None else d["k"],
+                                 d["temperature"], d["uniforms"], k_uniform=self.k_uniform,
                                  accepted_len=self.accepted, emitted_tokens=self.emitted,
                                  workspace=self.workspace, stream=self.stream)
 
 
+class L2Flush:
+    """Evicts the previous pass's lines from L2 by READING a buffer of twice the L2 size (a sum
+    over it).  Reading leaves clean lines behind; overwriting the buffer instead would leave the
+    L2 full of dirty lines whose write-back (126 MB) is then charged to the pass under test."""
+    def __init__(self, device):
+        import torch
+        self.buf = torch.zeros(2 * L2_BYTES // 4, dtype=torch.int32, device=device)
+        self.sink = torch.zeros(1, dtype=torch.int64, device=device)
+
+    def zero_(self):           # the name the timing loops call
+        import torch
+        torch.sum(self.buf.view(1, -1), dim=(1,), out=self.sink)
+
+
 def time_steps(dw, steps, warmup, flush=None, barrier=None):
-    """Mean ms per step over `steps` passes, CUDA events on the launching stream."""
+    """Mean ms per step over `steps` passes, CUDA events on the launching stream.  Without a
+    flush buffer the passes run back to back inside one event pair; with one, the buffer is
+    overwritten before every pass and each pass has its own event pair."""
+    return time_steps_stats(dw, steps, warmup, flush, barrier)["mean_ms"]
+
+
+def time_steps_stats(dw, steps, warmup, flush=None, barrier=None, per_step=True):
+    """{"mean_ms", "median_ms", "min_ms"}: the mean as time_steps states it; median and minimum from
+    per-pass event pairs (for back-to-back runs taken in a second loop of at most 200 passes)."""
     import torch
     for _ in range(warmup):
         if flush is not None:
@@ -197,6 +263,20 @@ def time_steps(dw, steps, warmup, flush=None, barrier=None):
     if barrier:
         barrier()
     torch.cuda.synchronize()
+
+    def each(n):
+        # all passes are enqueued at once, an event before and after each: the device-side time
+        # of every pass, without the host's launch latency in it
+        pairs = []
+        for _ in range(n):
+            if flush is not None:
+                flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); dw.step(); e1.record()
+            pairs.append((e0, e1))
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in pairs]
+
     if flush is None:
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -204,18 +284,36 @@ def time_steps(dw, steps, warmup, flush=None, barrier=None):
             dw.step()
         e1.record()
         torch.cuda.synchronize()
-        total = e0.elapsed_time(e1)
+        mean = e0.elapsed_time(e1) / steps
+        if barrier:
+            barrier()
+        singles = each(min(steps, 200)) if per_step else [mean]
     else:
-        total = 0.0
-        for _ in range(steps):
-            flush.zero_()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(); dw.step(); e1.record()
-            torch.cuda.synchronize()
-            total += e0.elapsed_time(e1)
-    if barrier:
-        barrier()
-    return total / steps
+        singles = each(steps)
+        mean = float(np.mean(singles))
+        if barrier:
+            barrier()
+    return {"mean_ms": mean, "median_ms": float(np.median(singles)), "min_ms": float(np.min(singles))}
+
+
+def sustained_run(dw, seconds, ms_estimate, sampler):
+    """Back-to-back passes for at least `seconds` inside ONE event pair, with the SM clock sampled
+    meanwhile: the figure under the power cap, beside the short-run one."""
+    import torch
+    n = int(max(50, np.ceil(seconds * 1e3 / ms_estimate)))
+    for _ in range(20):
+        dw.step()
+    torch.cuda.synchronize()
+    sampler.region(True, "sustained")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        dw.step()
+    e1.record()
+    torch.cuda.synchronize()
+    sampler.region(False)
+    total_ms = e0.elapsed_time(e1)
+    return n, total_ms
 
 
 def kernel_times(dw, steps, flush=None):
@@ -370,17 +468,20 @@ def run_ours(args):
 
     w = W.make_config(args.config)
     dw = DeviceWorkload(w, device)
-    small = w.logit_bytes <= 2 * L2_BYTES
-    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device) if small else None
+    flush_buf = L2Flush(device)
+    flush = flush_buf if needs_flush(w) else None
 
     sampler = ClockSampler(local)
     sampler.start()
     sampler.region(True)
     launches0 = binding.launch_count()
-    ms = time_steps(dw, args.steps, args.warmup, flush=flush, barrier=barrier)
+    timing = time_steps_stats(dw, args.steps, args.warmup, flush=flush, barrier=barrier, per_step=False)
     launches = binding.launch_count() - launches0
     launches_timed = launches * args.steps // (args.steps + args.warmup)
-    ms = sharding.max_over_ranks(ms, device)
+    ms = sharding.max_over_ranks(timing["mean_ms"], device)
+    sampler.region(False)
+    per_pass = time_steps_stats(dw, min(args.steps, 200), 0, flush=flush) if flush is None else timing
+    sampler.region(True)
     k_steps = min(args.steps, 50)
     k_ms = kernel_times(dw, k_steps, flush=flush)
 
@@ -408,9 +509,10 @@ def run_ours(args):
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
     e2e_ms = sharding.max_over_ranks(e2e_ms, device)
     sampler.region(False)
-    sampler.stop()
     h2d = sum(v.numel() * v.element_size() for v in pinned.values())
     d2h = acc_h.numel() * 4 + em_h.numel() * 4
+    del pinned, arena
+    torch.cuda.empty_cache()
 
     positions = w.n_draft_total * world
     peak, peak_kind = measured_peak_gbs()
@@ -423,6 +525,11 @@ def run_ours(args):
     traffic = (NCU_TRAFFIC["bytes_per_launch"]
                if ring and args.config == 5 and NCU_TRAFFIC["csrc_sha256"] == csrc_sha256() else None)
     achieved = w.logit_bytes / (stats_ms * 1e-3) / 1e9
+    # special-function work: one base-2 exponential per logit in the statistics kernel; in the resolve
+    # kernel one per element of every row a token is drawn from (two rows at a rejection, one otherwise)
+    elt = 4 if w.dtype == "f32" else 2
+    acc_now = dw.accepted.cpu().numpy()
+    resolve_rows = int(sum(2 if int(a) < int(k) else 1 for a, k in zip(acc_now, w.k_per_row)))
     line = {
         "metric": METRIC, "value": positions / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -433,29 +540,55 @@ def run_ours(args):
                 "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps},
         "gpu_launches": int(launches_timed),
         "roofline": {"bound": "hbm", "kernel": names[1], "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind,
+                     "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
+                     "traffic_note": ("extrapolated from the ncu capture summarised under profiles/ (" +
+                                      NCU_TRAFFIC["workload"] + ")") if traffic else
+                                     "null: the kernel sources differ from those the ncu capture under profiles/ was taken on",
+                     "peak_source": peak_kind + " copy bandwidth (read + write); a read-only stream can exceed it",
                      "kernel_ms": stats_ms, "bytes_per_launch": int(w.logit_bytes),
                      "whole_pass_frac": w.logit_bytes / (ms * 1e-3) / 1e9 / peak,
-                     "frac_of_8000_datasheet": achieved / 8000.0},
+                     "frac_of_8000_datasheet": achieved / 8000.0,
+                     "ex2_per_s": {names[1]: w.logit_bytes / elt / (k_ms[1] * 1e-3),
+                                   names[2]: resolve_rows * w.V / (k_ms[2] * 1e-3)}},
         "kernel_ms": {names[0]: k_ms[0], names[1]: k_ms[1], names[2]: k_ms[2]},
+        "per_pass": {"median_us": per_pass["median_ms"] * 1e3, "min_us": per_pass["min_ms"] * 1e3,
+                     "note": "one event pair per pass (the headline mean is one pair around all passes)"},
     }
 
-    if args.early_exit and rank == 0 and world == 1:
+    solo = rank == 0 and world == 1
+    if solo and not args.no_sustained:
+        n, total_ms = sustained_run(dw, args.sustained_seconds, ms, sampler)
+        sus_ms = total_ms / n
+        clk = sampler.region_summary("sustained")
+        line["sustained"] = {
+            "passes": n, "seconds": total_ms * 1e-3, "ms_per_step": sus_ms, "value": positions / (sus_ms * 1e-3),
+            "unit": UNIT, "whole_pass_frac": w.logit_bytes / (sus_ms * 1e-3) / 1e9 / peak,
+            "short_run_whole_pass_frac": w.logit_bytes / (ms * 1e-3) / 1e9 / peak, "clocks": clk,
+            "us_times_median_mhz": (sus_ms * 1e3 * clk["sm_mhz"]) if clk["sm_mhz"] else None,
+            "short_run_us_times_median_mhz": (ms * 1e3 * line["clocks"]["sm_mhz"]) if line["clocks"]["sm_mhz"] else None,
+            "note": "back-to-back passes inside one event pair; sw_power_cap is expected on a long run"}
+    sampler.stop()
+
+    if solo and not args.no_early_exit and ring:
         binding.set_early_exit(True)
-        ems = time_steps(dw, min(args.steps, 100), args.warmup, flush=flush)
+        ee = time_steps_stats(dw, min(args.steps, 100), args.warmup, flush=flush)
         binding.set_early_exit(False)
-        acc = dw.accepted.cpu().numpy()
-        needed = sum(2 * min(int(a) + 1, int(k)) + (1 if a == k else 0) for a, k in zip(acc, w.k_per_row))
-        line["early_exit"] = {"ms_per_step": ems, "value": positions / (ems * 1e-3), "unit": UNIT,
-                              "rows_needed_frac": needed / (2 * w.n_draft_total + w.B),
-                              "note": "rows after a sequence's first clear rejection are not read; same tokens"}
+        acc_ee = dw.accepted.cpu().numpy()
+        em_ee = dw.emitted.cpu().numpy()
         dw.step()
         torch.cuda.synchronize()
-    if args.tree and rank == 0 and world == 1:
+        same = bool(np.array_equal(acc_ee, dw.accepted.cpu().numpy()) and np.array_equal(em_ee, dw.emitted.cpu().numpy()))
+        needed = sum(2 * min(int(a) + 1, int(k)) + (1 if a == k else 0) for a, k in zip(acc_ee, w.k_per_row))
+        line["early_exit"] = {"ms_per_step": ee["mean_ms"], "median_us": ee["median_ms"] * 1e3, "min_us": ee["min_ms"] * 1e3,
+                              "value": positions / (ee["mean_ms"] * 1e-3), "unit": UNIT,
+                              "rows_needed_frac": needed / (2 * w.n_draft_total + w.B),
+                              "parity_sample": {"sequences": int(w.B), "identical_to_normal_mode": same},
+                              "note": "rows after a sequence's first clear rejection are not read; same tokens"}
+    if solo and not args.no_tree:
         line["tree"] = tree_leg(device, min(args.steps, 50), args.warmup, peak)
-    if rank == 0 and world == 1 and not args.no_greedy:
+    if solo and not args.no_greedy:
         line["greedy"] = greedy_leg(dw, w, device, min(args.steps, 100), args.warmup, flush, peak)
-    if rank == 0 and world == 1:
+    if solo:
         # verify the timed output against the oracle on a sample of sequences, and time the oracle
         import oracle
         cores = os.cpu_count() or 1
@@ -471,9 +604,19 @@ def run_ours(args):
         ora = oracle.spec_verify(sub.target_logits, sub.draft_logits, sub.draft_tokens, sub.k_per_row,
                                  sub.temperature, sub.uniforms, threads=cores)
         dt = time.perf_counter() - t0
+        # the same oracle on ONE thread, on a smaller sample (about 3 s)
+        n_one = int(min(n_seq, max(1, 3.0 / max(per_seq_core_s, 1e-6))))
+        one = w.take(0, n_one)
+        t0 = time.perf_counter()
+        oracle.spec_verify(one.target_logits, one.draft_logits, one.draft_tokens, one.k_per_row, one.temperature,
+                           one.uniforms, threads=1)
+        dt_one = time.perf_counter() - t0
         line["cpu_baseline"] = {"value": sub.n_draft_total / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"first {n_seq} of {w.B} sequences ({sub.n_draft_total} draft positions), "
-                                          f"{dt:.2f} s wall on {cores} threads"}
+                                          f"{dt:.2f} s wall on {cores} threads",
+                                "single_thread": {"value": one.n_draft_total / dt_one, "unit": UNIT, "cores": 1,
+                                                  "sample": f"first {n_one} sequences ({one.n_draft_total} draft "
+                                                            f"positions), {dt_one:.2f} s"}}
         acc = dw.accepted.cpu().numpy()[:n_seq]
         em = dw.emitted.cpu().numpy()
         mism = excused = 0
@@ -494,21 +637,28 @@ def run_ours(args):
             allc = {}
             for c in (1, 2, 3, 4, 5):
                 if c == args.config:
-                    allc[str(c)] = {"us_per_call": ms * 1e3, "positions_per_s": w.n_draft_total / (ms * 1e-3),
+                    allc[str(c)] = {"us_per_call": ms * 1e3, "median_us": per_pass["median_ms"] * 1e3,
+                                    "min_us": per_pass["min_ms"] * 1e3,
+                                    "positions_per_s": w.n_draft_total / (ms * 1e-3),
                                     "logit_gbs": w.logit_bytes / (ms * 1e-3) / 1e9,
-                                    "frac_of_peak": w.logit_bytes / (ms * 1e-3) / 1e9 / peak}
+                                    "frac_of_peak": w.logit_bytes / (ms * 1e-3) / 1e9 / peak,
+                                    "l2_flushed": flush is not None, "input_sets": input_sets(w)}
                     continue
                 del dw
                 torch.cuda.empty_cache()
                 wc = W.make_config(c)
                 dw = DeviceWorkload(wc, device)
-                fl = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device) if wc.logit_bytes <= 2 * L2_BYTES else None
-                m = time_steps(dw, 50, 5, flush=fl)
+                fl = flush_buf if needs_flush(wc) else None
+                t = time_steps_stats(dw, 60, 5, flush=fl)
                 km = kernel_times(dw, 20, flush=fl)
-                allc[str(c)] = {"us_per_call": m * 1e3, "positions_per_s": wc.n_draft_total / (m * 1e-3),
+                m = t["mean_ms"]
+                allc[str(c)] = {"us_per_call": m * 1e3, "median_us": t["median_ms"] * 1e3, "min_us": t["min_ms"] * 1e3,
+                                "positions_per_s": wc.n_draft_total / (m * 1e-3),
                                 "logit_gbs": wc.logit_bytes / (m * 1e-3) / 1e9,
                                 "frac_of_peak": wc.logit_bytes / (m * 1e-3) / 1e9 / peak,
                                 "kernel_us": [x * 1e3 for x in km], "l2_flushed": fl is not None,
+                                "input_sets": input_sets(wc),
+                                "k_per_row": "NULL (uniform lookahead)" if dw.k_uniform is not None else "device array",
                                 "graph_replay_us_no_flush": graph_replay_us(dw),
                                 "path": {1: "streaming", 2: "ring"}[binding.last_path()]}
             line["all_configs"] = allc
@@ -528,9 +678,11 @@ def main():
     ap.add_argument("--no-all-configs", action="store_true")
     ap.add_argument("--path", choices=["auto", "streaming", "ring"], default="auto")
     ap.add_argument("--no-greedy", action="store_true", help="skip the extra greedy-verification leg")
-    ap.add_argument("--tree", action="store_true", help="also time tree-structured verification (extra key)")
-    ap.add_argument("--early-exit", action="store_true",
-                    help="also time the optional early-exit mode (extra key; the headline stays the full pass)")
+    ap.add_argument("--no-tree", action="store_true", help="skip the tree-structured verification leg")
+    ap.add_argument("--no-early-exit", action="store_true",
+                    help="skip the leg that times the optional early-exit mode (the headline is always the full pass)")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the seconds-long back-to-back run")
+    ap.add_argument("--sustained-seconds", type=float, default=2.2)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

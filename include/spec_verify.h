@@ -314,8 +314,9 @@ size_t spec_verify_host_arena_bytes(int dtype, int32_t B, int64_t n_draft_total,
  * (pinned memory makes the copies asynchronous to the host but is not required);
  * `arena` is a DEVICE pointer, 256-byte aligned, of at least
  * spec_verify_host_arena_bytes(...) bytes, owned by the caller and clobbered.
- * Logits rows are copied with their pitch removed.  Errors as for spec_verify; a failed
- * copy or synchronisation returns SPECV_ERR_CUDA.
+ * Logits rows are copied with their pitch removed.  `flags` as for spec_verify_ex (0: automatic
+ * kernel set, normal mode).  Errors as for spec_verify_ex; a failed copy or synchronisation returns
+ * SPECV_ERR_CUDA.
  */
 int spec_verify_host(const void* target_logits, const void* draft_logits, int dtype,
                      int64_t V, int64_t ld_target, int64_t ld_draft,
@@ -325,7 +326,7 @@ int spec_verify_host(const void* target_logits, const void* draft_logits, int dt
                      const float* uniforms,
                      int32_t* accepted_len, int32_t* emitted_tokens, int32_t* row_status,
                      float* diag_p_tok, float* diag_q_tok,
-                     void* arena, size_t arena_bytes, void* cuda_stream);
+                     void* arena, size_t arena_bytes, void* cuda_stream, uint32_t flags);
 
 /*
  * spec_verify for callers that must not allocate device memory.  (No counterpart in the

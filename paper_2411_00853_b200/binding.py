@@ -52,7 +52,7 @@ def load() -> ctypes.CDLL:
     lib.spec_verify.restype = ctypes.c_int
     lib.spec_verify.argtypes = common
     lib.spec_verify_host.restype = ctypes.c_int
-    lib.spec_verify_host.argtypes = common
+    lib.spec_verify_host.argtypes = common + [ctypes.c_uint32]
     lib.spec_verify_noalloc.restype = ctypes.c_int
     lib.spec_verify_noalloc.argtypes = common[:-3] + [vp]
     lib.spec_verify_ex.restype = ctypes.c_int
@@ -269,7 +269,7 @@ def spec_verify_noalloc(target_logits, draft_logits, draft_tokens, k_per_row, te
 
 def spec_verify_host(target_logits, draft_logits, draft_tokens, k_per_row, temperature, uniforms, arena, *,
                      k_uniform=None, accepted_len=None, emitted_tokens=None, row_status=None,
-                     diag_p_tok=None, diag_q_tok=None, stream=None):
+                     diag_p_tok=None, diag_q_tok=None, stream=None, flags=None):
     """The same pass on HOST tensors (CPU torch tensors, ideally pinned); `arena` is a CUDA uint8
     tensor of at least host_arena_bytes(...) bytes.  Blocks until the outputs are on the host."""
     lib = load()
@@ -285,7 +285,8 @@ def spec_verify_host(target_logits, draft_logits, draft_tokens, k_per_row, tempe
                               V, ld_t, ld_d, _ptr(draft_tokens) if D else None, _ptr(k_per_row), B, k_uniform, D,
                               _ptr(temperature), per_row, _ptr(uniforms), _ptr(accepted_len), _ptr(emitted_tokens),
                               _ptr(row_status), _ptr(diag_p_tok), _ptr(diag_q_tok), _ptr(arena),
-                              arena.numel() * arena.element_size(), ctypes.c_void_p(stream))
+                              arena.numel() * arena.element_size(), ctypes.c_void_p(stream),
+                              _default_flags if flags is None else int(flags))
     _check(rc)
     return accepted_len, emitted_tokens
 

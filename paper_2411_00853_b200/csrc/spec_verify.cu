@@ -521,10 +521,11 @@ int spec_verify_host(const void* target_logits, const void* draft_logits, int dt
                      const int32_t* k_per_row, int32_t B, int32_t k_uniform, int64_t n_draft_total,
                      const float* temperature, int temperature_per_row, const float* uniforms,
                      int32_t* accepted_len, int32_t* emitted_tokens, int32_t* row_status, float* diag_p_tok,
-                     float* diag_q_tok, void* arena, size_t arena_bytes, void* cuda_stream) {
+                     float* diag_q_tok, void* arena, size_t arena_bytes, void* cuda_stream, uint32_t flags) {
     int rc = validate(target_logits, draft_logits, dtype, V, ld_target, ld_draft, draft_tokens, k_per_row, B,
                       k_uniform, n_draft_total, temperature, uniforms, accepted_len, emitted_tokens);
     if (rc != SPECV_OK) return rc;
+    if (!flags_ok(flags)) return SPECV_ERR_FLAGS;
     if (!arena) return SPECV_ERR_NULL;
     if (!aligned_to(arena, 256)) return SPECV_ERR_ALIGN;
     const Arena a = arena_layout(dtype, B, n_draft_total, V);
@@ -550,7 +551,7 @@ int spec_verify_host(const void* target_logits, const void* draft_logits, int dt
         !h2d(a.uniforms, uniforms, (size_t)(D + B) * 4))
         return SPECV_ERR_CUDA;
 
-    rc = spec_verify(base + a.target, D ? base + a.draft : nullptr, dtype, V, V, V,
+    rc = spec_verify_ex(base + a.target, D ? base + a.draft : nullptr, dtype, V, V, V,
                      D ? reinterpret_cast<const int32_t*>(base + a.tokens) : nullptr,
                      k_per_row ? reinterpret_cast<const int32_t*>(base + a.k) : nullptr, B, k_uniform, D,
                      reinterpret_cast<const float*>(base + a.temperature), temperature_per_row,
@@ -559,7 +560,7 @@ int spec_verify_host(const void* target_logits, const void* draft_logits, int dt
                      reinterpret_cast<int32_t*>(base + a.status),
                      diag_p_tok ? reinterpret_cast<float*>(base + a.diag_p) : nullptr,
                      diag_q_tok ? reinterpret_cast<float*>(base + a.diag_q) : nullptr, base + a.ws,
-                     arena_bytes - a.ws, stream);
+                     arena_bytes - a.ws, stream, flags, 0, 0, nullptr);
     if (rc != SPECV_OK) return rc;
 
     auto d2h = [&](void* dst, size_t at, size_t bytes) {

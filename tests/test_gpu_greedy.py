@@ -136,7 +136,7 @@ def test_argument_errors():
     def call(dtype=0, V=64, ld=64, B=1, k=3, D=3, target=t, ws_bytes=4096):
         return lib.spec_verify_greedy(target.data_ptr() if target is not None else None, dtype, V, ld, tok.data_ptr(),
                                       None, B, k, D, out.data_ptr(), out.data_ptr(), None, None, ws.data_ptr(),
-                                      ws_bytes, None)
+                                      ws_bytes, None, binding.default_flags() & 3)
     assert call() == 0
     assert call(dtype=3) == 3 and call(ld=63) == 2 and call(k=2) == 2 and call(target=None) == 1
     assert call(ws_bytes=16) == 5
