@@ -96,15 +96,14 @@ specv_ring_argmax(const char* __restrict__ target, int64_t pitch_t, int64_t V, i
     const int nck = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
     constexpr int kQuarterVecs = kChunkBytes / kWarpsPerChunk / 16;
 
-    if (tid == 0) {
-        ring_init(sh.ring);
-        for (int i = 0; i < kItemDepth; ++i) {
-            mbar_init(smem_u32(&sh.item_done[i]), kCWarps);
-            mbar_init(smem_u32(&sh.item_free[i]), 1);
-        }
+    ring_init(sh.ring, tid);
+    if (tid >= 32 && tid < 32 + kItemDepth) {
+        mbar_init(smem_u32(&sh.item_done[tid - 32]), kCWarps);
+        mbar_init(smem_u32(&sh.item_free[tid - 32]), 1);
+    } else if (tid == 64) {
         sh.err = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
     pdl_launch_dependents();
     // nothing the prologue writes is read here: the rows are the caller's; the wait for it sits

@@ -143,11 +143,12 @@ struct ChunkRing {
     signed char armed_parity[kRingSlots];       // parity of the last copy armed on a slot, -1: none
 };
 
-__device__ __forceinline__ void ring_init(ChunkRing& ring, int warps_per_chunk = kWarpsPerChunk) {
-    for (int s = 0; s < kRingSlots; ++s) {
-        mbar_init(smem_u32(&ring.full_bar[s]), 1);
-        mbar_init(smem_u32(&ring.empty_bar[s]), warps_per_chunk);
-        ring.armed_parity[s] = -1;
+// Called by every thread of the CTA (one slot per thread; a fence and a CTA barrier must follow).
+__device__ __forceinline__ void ring_init(ChunkRing& ring, int tid, int warps_per_chunk = kWarpsPerChunk) {
+    if (tid < kRingSlots) {
+        mbar_init(smem_u32(&ring.full_bar[tid]), 1);
+        mbar_init(smem_u32(&ring.empty_bar[tid]), warps_per_chunk);
+        ring.armed_parity[tid] = -1;
     }
 }
 
@@ -377,6 +378,20 @@ __device__ __forceinline__ void block_offsets(const BatchView& in, int32_t* off,
                                               int nthreads, bool publish, int32_t* seq_status, int32_t* done) {
     const int32_t* kp = in.k_per_row;
     const int32_t ku = in.k_uniform;
+    if (!kp) {
+        // every sequence has the same lookahead: no scan (the host has checked B * k_uniform == n_draft_total)
+        for (int32_t b = tid; b <= in.B; b += nthreads) {
+            const long long excl = (long long)b * ku;
+            off[b] = (int32_t)(excl < in.n_draft_total ? excl : in.n_draft_total);
+            if (publish && b < in.B) {
+                const float T = in.temperature[in.per_row_temperature ? b : 0];
+                seq_status[b] = (!(T > 0.0f) || isinf(T)) ? 2 : 0;          // SPECV_ROW_BAD_TEMPERATURE
+                done[b] = 0;
+            }
+        }
+        __syncthreads();
+        return;
+    }
     auto lookahead = [&](int32_t b) { const int32_t k = kp ? kp[b] : ku; return (long long)(k > 0 ? k : 0); };
     block_exclusive_prefix(lookahead, in.B, in.n_draft_total, off, warp_tot, tid, nthreads,
                            [&](int32_t b, long long excl) {
@@ -487,19 +502,18 @@ specv_ring_stats(BatchView in, RingScratch ws, int prologue_too) {
     const int64_t row_bytes = in.V * E::kBytes;
     const int nck = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
 
-    if (tid == 0) {
-        ring_init(sh.ring, kStatsWarpsPerChunk);
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&sh.batch_full[i]), 1);
-            mbar_init(smem_u32(&sh.batch_empty[i]), kCWarps + 1);   // statistics warps, merge warp
-        }
-        for (int i = 0; i < kItemDepth; ++i) {
-            mbar_init(smem_u32(&sh.item_done[i]), kCWarps);
-            mbar_init(smem_u32(&sh.item_free[i]), 1);
-        }
+    // barriers: one thread each (the scan of the lookahead lengths below holds the CTA barrier that follows)
+    ring_init(sh.ring, tid, kStatsWarpsPerChunk);
+    if (tid >= 32 && tid < 34) {
+        mbar_init(smem_u32(&sh.batch_full[tid - 32]), 1);
+        mbar_init(smem_u32(&sh.batch_empty[tid - 32]), kCWarps + 1);   // statistics warps, merge warp
+    } else if (tid >= 64 && tid < 64 + kItemDepth) {
+        mbar_init(smem_u32(&sh.item_done[tid - 64]), kCWarps);
+        mbar_init(smem_u32(&sh.item_free[tid - 64]), 1);
+    } else if (tid == 96) {
         sh.err = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     pdl_launch_dependents();       // the next kernel may move in as SMs free up
     // Nothing a prologue kernel writes is needed here: every CTA scans the lookahead lengths
     // itself.  Only a tree batch has to wait -- the flags of contexts with children come from the
@@ -932,19 +946,17 @@ specv_ring_resolve(BatchView in, RingScratch ws, int32_t* __restrict__ accepted_
     const int32_t nvec_row = (int32_t)(row_bytes / 16);
     const int32_t nseg = (int32_t)((in.V + SEG - 1) / SEG);
 
-    if (tid == 0) {
-        ring_init(sh.ring);
-        for (int i = 0; i < kPartDepth; ++i) {
-            mbar_init(smem_u32(&sh.rec_full[i]), 1);
-            mbar_init(smem_u32(&sh.rec_empty[i]), kCWarps + 2);   // consumers, copy warp, locator
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&sh.seg_done[i]), kCWarps);
-            mbar_init(smem_u32(&sh.seg_free[i]), 1);
-        }
+    ring_init(sh.ring, tid);
+    if (tid >= 32 && tid < 32 + kPartDepth) {
+        mbar_init(smem_u32(&sh.rec_full[tid - 32]), 1);
+        mbar_init(smem_u32(&sh.rec_empty[tid - 32]), kCWarps + 2);   // consumers, copy warp, locator
+    } else if (tid >= 64 && tid < 66) {
+        mbar_init(smem_u32(&sh.seg_done[tid - 64]), kCWarps);
+        mbar_init(smem_u32(&sh.seg_free[tid - 64]), 1);
+    } else if (tid == 96) {
         sh.err = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     block_offsets(in, sh.off, sh.warp_tot, tid, kRingResolveThreads, false, nullptr, nullptr);
 
     const int64_t total = (int64_t)in.B * nck;
@@ -1218,20 +1230,18 @@ specv_ring_stats_early(BatchView in, RingScratch ws) {
     const int64_t row_bytes = in.V * E::kBytes;
     const int nck = (int)((row_bytes + kChunkBytes - 1) / kChunkBytes);
 
-    if (tid == 0) {
-        ring_init(sh.ring, kStatsWarpsPerChunk);
-        for (int i = 0; i < kEarlyDescDepth; ++i) {
-            mbar_init(smem_u32(&sh.desc_full[i]), 1);
-            mbar_init(smem_u32(&sh.desc_empty[i]), 1 + kCWarps + 1);   // copy warp, statistics warps, merge warp
-        }
-        for (int i = 0; i < kItemDepth; ++i) {
-            mbar_init(smem_u32(&sh.item_go[i]), 1);
-            mbar_init(smem_u32(&sh.item_done[i]), kCWarps);
-            mbar_init(smem_u32(&sh.item_free[i]), 1);
-        }
+    ring_init(sh.ring, tid, kStatsWarpsPerChunk);
+    if (tid >= 32 && tid < 32 + kEarlyDescDepth) {
+        mbar_init(smem_u32(&sh.desc_full[tid - 32]), 1);
+        mbar_init(smem_u32(&sh.desc_empty[tid - 32]), 1 + kCWarps + 1);   // copy warp, statistics warps, merge warp
+    } else if (tid >= 64 && tid < 64 + kItemDepth) {
+        mbar_init(smem_u32(&sh.item_go[tid - 64]), 1);
+        mbar_init(smem_u32(&sh.item_done[tid - 64]), kCWarps);
+        mbar_init(smem_u32(&sh.item_free[tid - 64]), 1);
+    } else if (tid == 96) {
         sh.err = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
     pdl_wait_for_predecessor();    // the work list
     pdl_launch_dependents();
