@@ -300,6 +300,30 @@ int spec_verify_greedy(const void* target_logits, int dtype, int64_t V, int64_t 
                        void* workspace, size_t workspace_bytes, void* cuda_stream, uint32_t flags);
 
 /*
+ * Self-test of the bounded waits (a diagnostic; the paper has no counterpart).  Every wait inside
+ * the ring kernels -- on a shared-memory barrier that a bulk copy or another warp completes --
+ * carries a limit of about a second; past it the wait gives up, records which wait it was, every
+ * other wait of the thread block returns at once, and the kernel ends in bounds with
+ * SPECV_ROW_INTERNAL in row_status.  This entry point runs that mechanism on purpose, harmlessly:
+ * one small kernel whose first warp waits, with the given limit, on a barrier that nothing ever
+ * completes.  out4 is a DEVICE array of four int64: [0] the error word (77: the first wait gave
+ * up), [1] clock cycles the first wait lasted (just over the limit), [2] cycles of a second wait
+ * on another barrier (a few hundred: it returns because the block has already failed), [3] 1 once
+ * the kernel has reached its end.  limit_cycles in [1, 2e9]; else SPECV_ERR_SHAPE.
+ */
+int spec_verify_selftest_bounded_wait(int64_t limit_cycles, int64_t* out4, void* cuda_stream);
+
+/*
+ * Debug aid (the paper has no counterpart).  A library built with -DSPECV_DEBUG
+ * (python -m paper_2411_00853_b200.build --debug -> libspecverify_debug.so) range-checks every row
+ * index, split number, segment number and token id that the streaming kernels compute, before use;
+ * a violation is recorded and the access skipped, nothing traps.  Returns the largest site code
+ * recorded on the current device since the library was loaded (0: none; waits for the device),
+ * -1 from a library built without the checks, -2 if the value could not be read.
+ */
+int spec_verify_debug_violation(void);
+
+/*
  * Bytes of device memory ("arena") that spec_verify_host needs: device copies of all
  * inputs and outputs with dense pitch (ld = V) plus the workspace.  0 for arguments that
  * would be rejected.

@@ -24,6 +24,10 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "spec_verify_oracle.c")
 _LIB = os.path.join(_HERE, "liboracle.so")
+_LIB_SAN = os.path.join(_HERE, "liboracle_san.so")
+# ORACLE_SANITIZE=1: load the build instrumented with AddressSanitizer and
+# UndefinedBehaviorSanitizer (the process must have libasan preloaded)
+_SANITIZE = os.environ.get("ORACLE_SANITIZE", "") not in ("", "0")
 
 F32 = 0
 BF16 = 1
@@ -36,16 +40,19 @@ ROW_ZERO_RESIDUAL = 8
 ROW_BAD_PARENT = 32
 
 
-def build(force: bool = False) -> str:
-    """Compile the C oracle with gcc (no fast-math, no FMA contraction)."""
-    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+def build(force: bool = False, sanitize: bool = False) -> str:
+    """Compile the C oracle with gcc (no fast-math, no FMA contraction).  sanitize: the build
+    with -fsanitize=address,undefined (same arithmetic flags)."""
+    lib = _LIB_SAN if sanitize else _LIB
+    stale = (not os.path.exists(lib)) or os.path.getmtime(lib) < os.path.getmtime(_SRC)
     if force or stale:
-        tmp = _LIB + f".{os.getpid()}.tmp"
+        tmp = lib + f".{os.getpid()}.tmp"
+        extra = ["-fsanitize=address,undefined", "-fno-omit-frame-pointer", "-g"] if sanitize else []
         subprocess.check_call(
-            ["gcc", "-std=c99", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
+            ["gcc", "-std=c99", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared", *extra,
              "-o", tmp, _SRC, "-lm"])
-        os.replace(tmp, _LIB)
-    return _LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 _lib = None
@@ -54,7 +61,7 @@ _lib = None
 def _load():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(build())
+        lib = ctypes.CDLL(build(sanitize=_SANITIZE))
         vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
         lib.oracle_spec_verify.restype = ctypes.c_int
         lib.oracle_spec_verify.argtypes = [

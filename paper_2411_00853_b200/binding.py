@@ -13,7 +13,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libspecverify.so")
+# SPECV_LIB names another build of the same library (the debug or the sanitizer build)
+LIB_PATH = os.environ.get("SPECV_LIB") or os.path.join(_HERE, "libspecverify.so")
 
 F32, BF16, F16 = 0, 1, 2
 ROW_BAD_K, ROW_BAD_TEMPERATURE, ROW_BAD_TOKEN, ROW_ZERO_RESIDUAL = 1, 2, 4, 8
@@ -22,7 +23,8 @@ ROW_INTERNAL, ROW_BAD_PARENT = 16, 32
 EXPORTS = ("spec_verify", "spec_verify_host", "spec_verify_workspace_bytes",
            "spec_verify_host_arena_bytes", "spec_verify_strerror", "spec_verify_last_cuda_error",
            "spec_verify_launch_count", "spec_verify_set_trace_events", "spec_verify_noalloc", "spec_verify_ex",
-           "spec_verify_last_path", "spec_verify_next_lookahead",
+           "spec_verify_last_path", "spec_verify_next_lookahead", "spec_verify_selftest_bounded_wait",
+           "spec_verify_debug_violation",
            "spec_verify_greedy", "spec_verify_greedy_workspace_bytes",
            "spec_verify_tree", "spec_verify_tree_workspace_bytes")
 NOALLOC_SCRATCH_BYTES = 4 << 20
@@ -69,8 +71,12 @@ def load() -> ctypes.CDLL:
                                        ctypes.c_uint32]
     lib.spec_verify_greedy_workspace_bytes.restype = sz
     lib.spec_verify_greedy_workspace_bytes.argtypes = [i32, i64]
+    lib.spec_verify_selftest_bounded_wait.restype = ctypes.c_int
+    lib.spec_verify_selftest_bounded_wait.argtypes = [i64, vp, vp]
     lib.spec_verify_last_path.restype = ctypes.c_int
     lib.spec_verify_last_path.argtypes = []
+    lib.spec_verify_debug_violation.restype = ctypes.c_int
+    lib.spec_verify_debug_violation.argtypes = []
     lib.spec_verify_workspace_bytes.restype = sz
     lib.spec_verify_workspace_bytes.argtypes = [i32, i64, i64]
     lib.spec_verify_host_arena_bytes.restype = sz
@@ -150,6 +156,22 @@ def next_lookahead(k_per_row, accepted_len, k_min: int, k_max: int, *, k_uniform
     _check(load().spec_verify_next_lookahead(_ptr(k_per_row), int(k_uniform), _ptr(accepted_len), B, int(k_min),
                                              int(k_max), _ptr(out), ctypes.c_void_p(stream)))
     return out
+
+
+def selftest_bounded_wait(limit_cycles: int, stream=None):
+    """Runs the library's bounded wait into its limit on purpose (see the header).  Returns
+    (error_word, cycles_first_wait, cycles_second_wait, reached_end) as Python ints."""
+    out = torch.zeros(4, dtype=torch.int64, device="cuda")
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(load().spec_verify_selftest_bounded_wait(int(limit_cycles), _ptr(out), ctypes.c_void_p(stream)))
+    torch.cuda.synchronize()
+    return tuple(int(v) for v in out.cpu())
+
+
+def debug_violation() -> int:
+    """Largest range-check site code recorded by a -DSPECV_DEBUG build (0: none; -1: not such a build)."""
+    return int(load().spec_verify_debug_violation())
 
 
 def last_path() -> int:

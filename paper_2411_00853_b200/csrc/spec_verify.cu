@@ -959,3 +959,29 @@ extern "C" int spec_verify_noalloc(const void* target_logits, const void* draft_
                     row_status, diag_p_tok, diag_q_tok, scratch, 0u, 0, 0, nullptr,
                     static_cast<cudaStream_t>(cuda_stream));
 }
+
+// ---------------------------------------------------------------------------------
+// Self-test of the bounded waits
+// ---------------------------------------------------------------------------------
+extern "C" int spec_verify_selftest_bounded_wait(int64_t limit_cycles, int64_t* out4, void* cuda_stream) {
+    if (!out4) return SPECV_ERR_NULL;
+    if (limit_cycles < 1 || limit_cycles > 2000000000LL) return SPECV_ERR_SHAPE;
+    if (!aligned_to(out4, 8)) return SPECV_ERR_ALIGN;
+    specv::specv_selftest_bounded_wait<<<1, 64, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        (long long)limit_cycles, reinterpret_cast<long long*>(out4));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cuda_ok(cudaGetLastError()) ? SPECV_OK : SPECV_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------
+// Debug build: the recorded range violation
+// ---------------------------------------------------------------------------------
+extern "C" int spec_verify_debug_violation(void) {
+#ifdef SPECV_DEBUG
+    int v = 0;
+    if (!cuda_ok(cudaMemcpyFromSymbol(&v, specv::g_debug_violation, sizeof(int)))) return -2;
+    return v;
+#else
+    return -1;
+#endif
+}

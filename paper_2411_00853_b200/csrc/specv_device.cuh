@@ -16,6 +16,20 @@ constexpr int kF16 = 2;
 // Finite stand-in for "no maximum seen yet".  Finite so that (-inf logit) - reference
 // is -inf, never NaN: masked logits (-inf) then contribute exactly 0.
 constexpr float kNoMax = -3.0e38f;
+
+// Debug build (-DSPECV_DEBUG): every row index and token id the streaming kernels compute is
+// range-checked before it is used; a violation is recorded (the largest site code seen, readable
+// through spec_verify_debug_violation) and the access is skipped -- nothing traps.  In the normal
+// build the checks compile to nothing.
+#ifdef SPECV_DEBUG
+__device__ int g_debug_violation = 0;
+__device__ __forceinline__ bool debug_in_range(bool ok, int site) {
+    if (!ok) atomicMax(&g_debug_violation, site);
+    return ok;
+}
+#else
+__device__ __forceinline__ bool debug_in_range(bool, int) { return true; }
+#endif
 constexpr double kLog2e = 1.4426950408889634074;
 
 __device__ __forceinline__ float ex2_approx(float x) {

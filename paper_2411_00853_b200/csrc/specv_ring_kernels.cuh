@@ -109,13 +109,47 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // A parity wait is only sound while the barrier is at most one phase ahead of the waiter;
 // every barrier below is used so that its next phase cannot complete before all waiters of
 // the current one are through.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* err, int site) {
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* err, int site,
+                                          long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         if (*err) return;
-        if (clock64() - t0 > kWaitLimitCycles) { *err = site; return; }
+        if (clock64() - t0 > limit_cycles) { *err = site; return; }
     }
+}
+
+// Self-test of the bounded wait (spec_verify_selftest_bounded_wait): one warp waits on a barrier
+// that nothing ever completes, with a short limit.  The wait must give up, name itself in the
+// error word, and every later wait of the CTA must return at once; the kernel ends normally.
+// out[0]: error word, out[1]: clock cycles the first wait took, out[2]: cycles of a second wait,
+// out[3]: 1 once the end of the kernel is reached.
+__global__ void specv_selftest_bounded_wait(long long limit_cycles, long long* out) {
+    __shared__ unsigned long long never[2];
+    __shared__ int err_word;
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&never[0]), 1);
+        mbar_init(smem_u32(&never[1]), 1);
+        err_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    volatile int* err = &err_word;
+    const long long t0 = clock64();
+    mbar_wait(smem_u32(&never[0]), 0, err, 77, limit_cycles);      // phase 0 never completes
+    const long long t1 = clock64();
+    __syncwarp();
+    mbar_wait(smem_u32(&never[1]), 0, err, 78, limit_cycles);      // another barrier: returns because the CTA has failed
+    const long long t2 = clock64();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        out[0] = err_word;
+        out[1] = t1 - t0;
+        out[2] = t2 - t1;
+        out[3] = 1;
+    }
+    (void)lane;
 }
 // Plain bulk copy global -> this CTA's shared memory, completion on this CTA's mbarrier.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {

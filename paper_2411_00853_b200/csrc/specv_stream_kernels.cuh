@@ -162,6 +162,9 @@ specv_row_stats(BatchView in, const int32_t* __restrict__ off_d, int64_t n_targe
         const int64_t row = item / splits;
         const int split = (int)(item - row * splits);
         const bool is_target = row < n_target_rows;
+        if (!debug_in_range(row >= 0 && row < n_rows && split >= 0 && split < splits &&
+                                (is_target || row - n_target_rows < in.n_draft_total), 101))
+            continue;
         if (!is_target && in.ctx_has_children && !in.ctx_has_children[row - n_target_rows]) continue;   // block-uniform
         const char* rp = is_target ? in.target + row * in.pitch_t
                                    : in.draft + (row - n_target_rows) * in.pitch_d;
@@ -345,6 +348,7 @@ __device__ int32_t locate_in_segments(const SampleRows& sr, int64_t V, double u,
         }
         found_seg = __shfl_sync(0xffffffffu, found_seg, owner);
         base = shfl_double(base, owner);
+        if (!debug_in_range(found_seg >= 0 && found_seg < nseg, 104)) return -1;
         // inside the segment: recompute the masses exactly as pass A did
         float r[N];
         masses((int64_t)found_seg * 32 + lane, r);
@@ -466,6 +470,9 @@ specv_resolve(BatchView in, const int32_t* __restrict__ off_d, const int32_t* __
     int status = seq_status[b];
     const int32_t k_raw = in.k_per_row ? in.k_per_row[b] : in.k_uniform;
     const int32_t K = k_raw > 0 ? k_raw : 0;
+    // a valid sequence's rows lie inside the packed buffers
+    if (!(status & 1) && !debug_in_range(d0 >= 0 && d0 + K <= in.n_draft_total && t0 + K < n_target_rows, 102))
+        status |= 16;
 
     if (tid == 0) { first_reject = K; bad_token = 0; }
     __syncthreads();
@@ -543,6 +550,7 @@ specv_resolve(BatchView in, const int32_t* __restrict__ off_d, const int32_t* __
         token = block_inverse_cdf<DT, kResolveWarps, false>(sr, in.V, u2, seg, &result_slot, tid >> 5, sync_all);
     }
     if (token < 0) token = (int32_t)(in.V - 1);   // a row without any mass (all logits -inf)
+    if (!debug_in_range(token >= 0 && (int64_t)token < in.V && n >= 0 && n <= K, 103)) token = -1;
 
     for (int32_t i = tid; i <= K; i += kResolveThreads)
         emitted[t0 + i] = (i < n) ? in.tokens[d0 + i] : (i == n ? token : -1);
