@@ -300,6 +300,47 @@ int spec_verify_greedy(const void* target_logits, int dtype, int64_t V, int64_t 
                        void* workspace, size_t workspace_bytes, void* cuda_stream, uint32_t flags);
 
 /*
+ * The verify pass fed with HIDDEN STATES instead of logits: the step in front of it fused with its
+ * first half.  The paper's section "Speculative Sampling Results" has the target model score the
+ * drafted positions in one parallel pass (and the draft model before it); the output of those passes
+ * -- logits = hidden x weight^T of each model's output layer -- is what the verify pass reads.
+ * Here the two products run on the tensor cores (bf16 inputs, fp32 accumulation, results rounded to
+ * bf16) and the row statistics of the verify pass -- (reference, sum) of 2^(logit * log2(e)/T - reference)
+ * over the vocabulary, taken from the ROUNDED logits -- are computed in the products' epilogue, while
+ * the accumulators are still on chip.  The logits are written once, to the caller's buffers (the
+ * resolve step reads the one or two rows per sequence a token is drawn from, and the caller may want
+ * them), and never read back for the statistics.  Results are those of spec_verify on the logits
+ * this call writes (ring kernels).
+ *
+ *   target_hidden  bf16 [n_draft_total + B, ld_th]  hidden state of every target row (packing of target_logits)
+ *   target_weight  bf16 [V, ld_tw]                  output-layer weight of the target model, row v = token v
+ *   draft_hidden   bf16 [n_draft_total, ld_dh], draft_weight bf16 [V, ld_dw]   the same for the draft model
+ *   H_target, H_draft                               hidden sizes (>= 1); ld_* >= H in elements
+ *   target_logits  out, bf16 [n_draft_total + B, ld_target];  draft_logits out, bf16 [n_draft_total, ld_draft]
+ * All four inputs: DEVICE pointers on 16-byte boundaries with pitches that are multiples of 16 bytes
+ * (tensor-map loads); the logits buffers as the ring kernels want them (rows on 16-byte boundaries,
+ * V * 2 a multiple of 16, V <= 2^19, B <= 4095) -- else SPECV_ERR_SHAPE.  Everything else
+ * (draft_tokens .. diag_q_tok, asynchrony, error reporting) as for spec_verify;
+ * workspace >= spec_verify_from_hidden_workspace_bytes(B, n_draft_total, V).
+ * spec_verify_from_hidden_status reads back (after waiting for cuda_stream) the status word of the
+ * product kernels of the last call on that workspace: 0, or the code of a bounded wait that expired.
+ */
+size_t spec_verify_from_hidden_workspace_bytes(int32_t B, int64_t n_draft_total, int64_t V);
+int spec_verify_from_hidden(const void* target_hidden, int64_t ld_th, int64_t H_target,
+                            const void* target_weight, int64_t ld_tw,
+                            const void* draft_hidden, int64_t ld_dh, int64_t H_draft,
+                            const void* draft_weight, int64_t ld_dw, int64_t V,
+                            void* target_logits, int64_t ld_target, void* draft_logits, int64_t ld_draft,
+                            const int32_t* draft_tokens, const int32_t* k_per_row,
+                            int32_t B, int32_t k_uniform, int64_t n_draft_total,
+                            const float* temperature, int temperature_per_row, const float* uniforms,
+                            int32_t* accepted_len, int32_t* emitted_tokens, int32_t* row_status,
+                            float* diag_p_tok, float* diag_q_tok,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+int spec_verify_from_hidden_status(const void* workspace, int32_t B, int64_t n_draft_total, int64_t V,
+                                   void* cuda_stream);
+
+/*
  * Self-test of the bounded waits (a diagnostic; the paper has no counterpart).  Every wait inside
  * the ring kernels -- on a shared-memory barrier that a bulk copy or another warp completes --
  * carries a limit of about a second; past it the wait gives up, records which wait it was, every

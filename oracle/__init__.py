@@ -76,6 +76,8 @@ def _load():
         lib.oracle_spec_verify_tree.argtypes = [
             vp, vp, ctypes.c_int, i64, i64, i64, vp, vp, vp, i32, i32, i64, vp, ctypes.c_int, vp,
             i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.oracle_lm_head.restype = None
+        lib.oracle_lm_head.argtypes = [vp, i64, vp, i64, i64, i64, i64, i64, i64, vp, i64]
         lib.oracle_spec_verify_greedy.restype = None
         lib.oracle_spec_verify_greedy.argtypes = [
             vp, ctypes.c_int, i64, i64, vp, vp, i32, i32, i64, i32, i32, vp, vp, vp, vp]
@@ -312,3 +314,27 @@ def spec_verify_tree(target_logits, draft_logits, node_tokens, node_parent, n_pe
         with ThreadPoolExecutor(max_workers=threads) as pool:
             list(pool.map(lambda k: run(int(edges[k]), int(edges[k + 1])), range(len(edges) - 1)))
     return res
+
+
+def lm_head(hidden: np.ndarray, weight: np.ndarray, *, threads: int = 1) -> np.ndarray:
+    """logits = hidden @ weight.T for bf16 bit patterns (uint16 arrays [M, H] and [V, H]): products
+    summed in double, one rounding to bf16.  Returns uint16 [M, V]."""
+    lib = _load()
+    h = np.ascontiguousarray(hidden, dtype=np.uint16)
+    w = np.ascontiguousarray(weight, dtype=np.uint16)
+    M, H = h.shape
+    V = w.shape[0]
+    assert w.shape[1] == H
+    out = np.zeros((M, V), np.uint16)
+
+    def run(r0, r1):
+        lib.oracle_lm_head(_ptr(h), H, _ptr(w), H, M, V, H, r0, r1, _ptr(out), V)
+
+    threads = max(1, min(int(threads), M))
+    if threads == 1:
+        run(0, M)
+    else:
+        edges = np.linspace(0, M, min(M, threads * 4) + 1).astype(int)
+        with ThreadPoolExecutor(max_workers=threads) as pool:
+            list(pool.map(lambda k: run(int(edges[k]), int(edges[k + 1])), range(len(edges) - 1)))
+    return out

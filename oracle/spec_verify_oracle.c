@@ -530,3 +530,49 @@ int oracle_spec_verify_tree(const void *target_logits, const void *draft_logits,
     free(p); free(q); free(r);
     return 0;
 }
+
+
+/*
+ * LM-head product in front of the verify pass (the paper's section "Speculative Sampling Results":
+ * the target model scores the drafted positions in one parallel pass; these logits are what the
+ * verify pass reads):  logits[r][v] = sum_k hidden[r][k] * weight[v][k], hidden and weight in bf16,
+ * the sum taken in double over k in index order, the result rounded once to bf16 (to nearest, ties
+ * to even).  Rows r in [r_begin, r_end).  All arrays are bf16 bit patterns.
+ * parity status: pinned by tests/test_oracle_lm_head.py (numpy's matmul on exactly representable
+ * inputs, hand-checked rounding cases).
+ */
+static uint16_t double_to_bf16_bits(double x)
+{
+    float f = (float)x;                 /* not exact in general: handled below */
+    /* round the DOUBLE to 8 significant bits directly: scale so that the bf16 ulp is 1 */
+    if (x == 0.0 || isnan(x) || isinf(x)) {
+        uint32_t b; memcpy(&b, &f, 4); return (uint16_t)(b >> 16);
+    }
+    int e;
+    double m = frexp(fabs(x), &e);       /* |x| = m * 2^e, m in [0.5, 1) */
+    if (e < -125) {                      /* bf16 subnormal range: ulp fixed at 2^-133 */
+        double q = nearbyint(ldexp(fabs(x), 133));
+        double r = ldexp(q, -133);
+        f = (float)(x < 0 ? -r : r);
+    } else {
+        double q = nearbyint(ldexp(m, 8)); /* 8 significant bits, ties to even (default rounding mode) */
+        double r = ldexp(q, e - 8);
+        f = (float)(x < 0 ? -r : r);     /* exact: r has 8 significant bits */
+    }
+    uint32_t b; memcpy(&b, &f, 4);
+    return (uint16_t)(b >> 16);
+}
+
+void oracle_lm_head(const uint16_t *hidden, int64_t ld_h, const uint16_t *weight, int64_t ld_w,
+                    int64_t M, int64_t V, int64_t H, int64_t r_begin, int64_t r_end,
+                    uint16_t *logits, int64_t ld_out)
+{
+    (void)M;
+    for (int64_t r = r_begin; r < r_end; ++r)
+        for (int64_t v = 0; v < V; ++v) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < H; ++k)
+                acc += logit_at(hidden + r * ld_h, ORACLE_BF16, k) * logit_at(weight + v * ld_w, ORACLE_BF16, k);
+            logits[r * ld_out + v] = double_to_bf16_bits(acc);
+        }
+}

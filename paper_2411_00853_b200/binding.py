@@ -24,7 +24,8 @@ EXPORTS = ("spec_verify", "spec_verify_host", "spec_verify_workspace_bytes",
            "spec_verify_host_arena_bytes", "spec_verify_strerror", "spec_verify_last_cuda_error",
            "spec_verify_launch_count", "spec_verify_set_trace_events", "spec_verify_noalloc", "spec_verify_ex",
            "spec_verify_last_path", "spec_verify_next_lookahead", "spec_verify_selftest_bounded_wait",
-           "spec_verify_debug_violation",
+           "spec_verify_debug_violation", "spec_verify_from_hidden", "spec_verify_from_hidden_workspace_bytes",
+           "spec_verify_from_hidden_status",
            "spec_verify_greedy", "spec_verify_greedy_workspace_bytes",
            "spec_verify_tree", "spec_verify_tree_workspace_bytes")
 NOALLOC_SCRATCH_BYTES = 4 << 20
@@ -75,6 +76,13 @@ def load() -> ctypes.CDLL:
     lib.spec_verify_selftest_bounded_wait.argtypes = [i64, vp, vp]
     lib.spec_verify_last_path.restype = ctypes.c_int
     lib.spec_verify_last_path.argtypes = []
+    lib.spec_verify_from_hidden_workspace_bytes.restype = sz
+    lib.spec_verify_from_hidden_workspace_bytes.argtypes = [i32, i64, i64]
+    lib.spec_verify_from_hidden.restype = ctypes.c_int
+    lib.spec_verify_from_hidden.argtypes = [vp, i64, i64, vp, i64, vp, i64, i64, vp, i64, i64, vp, i64, vp, i64, vp, vp, i32,
+                                            i32, i64, vp, ctypes.c_int, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.spec_verify_from_hidden_status.restype = ctypes.c_int
+    lib.spec_verify_from_hidden_status.argtypes = [vp, i32, i64, i64, vp]
     lib.spec_verify_debug_violation.restype = ctypes.c_int
     lib.spec_verify_debug_violation.argtypes = []
     lib.spec_verify_workspace_bytes.restype = sz
@@ -387,3 +395,55 @@ def spec_verify_tree(target_logits, draft_logits, node_tokens, node_parent, n_pe
                               _path_flags(flags))
     _check(rc)
     return accepted_len, emitted_tokens
+
+
+def from_hidden_workspace_bytes(B: int, n_draft_total: int, V: int) -> int:
+    return int(load().spec_verify_from_hidden_workspace_bytes(B, n_draft_total, V))
+
+
+def spec_verify_from_hidden(target_hidden, target_weight, draft_hidden, draft_weight, draft_tokens, k_per_row,
+                            temperature, uniforms, *, k_uniform=None, target_logits=None, draft_logits=None,
+                            accepted_len=None, emitted_tokens=None, row_status=None, diag_p_tok=None,
+                            diag_q_tok=None, workspace=None, stream=None):
+    """The verify pass from hidden states (bf16 CUDA tensors): target_hidden [sum(K)+B, H], target_weight
+    [V, H], draft_hidden [sum(K), Hd], draft_weight [V, Hd].  The logits (bf16) are written to
+    target_logits / draft_logits.  Returns (accepted_len, emitted_tokens, target_logits, draft_logits)."""
+    lib = load()
+    dev = target_hidden.device
+    V = target_weight.shape[0]
+    D = 0 if draft_hidden is None else draft_hidden.shape[0]
+    if k_per_row is None:
+        B = target_hidden.shape[0] - D
+        k_uniform = (D // B if B > 0 else 0) if k_uniform is None else k_uniform
+    else:
+        B, k_uniform = k_per_row.shape[0], 0
+    if target_logits is None:
+        target_logits = torch.empty((D + B, V), dtype=torch.bfloat16, device=dev)
+    if draft_logits is None:
+        draft_logits = torch.empty((max(D, 1), V), dtype=torch.bfloat16, device=dev)[:D]
+    if accepted_len is None:
+        accepted_len = torch.empty(B, dtype=torch.int32, device=dev)
+    if emitted_tokens is None:
+        emitted_tokens = torch.empty(D + B, dtype=torch.int32, device=dev)
+    if workspace is None:
+        workspace = _temporary_workspace(from_hidden_workspace_bytes(B, D, V), dev, stream)
+    if stream is None:
+        stream = torch.cuda.current_stream(dev).cuda_stream
+    per_row = int(temperature.numel() == B and B > 1)
+    ld = lambda t: t.stride(0) if t.shape[0] > 1 else max(t.shape[1], t.stride(0))
+    rc = lib.spec_verify_from_hidden(
+        _ptr(target_hidden), ld(target_hidden), target_hidden.shape[1], _ptr(target_weight), ld(target_weight),
+        _ptr(draft_hidden) if D else None, ld(draft_hidden) if D else 0, draft_hidden.shape[1] if D else 0,
+        _ptr(draft_weight) if D else None, ld(draft_weight) if D else 0, V,
+        _ptr(target_logits), ld(target_logits), _ptr(draft_logits) if D else None, ld(draft_logits) if D else V,
+        _ptr(draft_tokens) if D else None, _ptr(k_per_row), B, int(k_uniform), D, _ptr(temperature), per_row,
+        _ptr(uniforms), _ptr(accepted_len), _ptr(emitted_tokens), _ptr(row_status), _ptr(diag_p_tok), _ptr(diag_q_tok),
+        _ptr(workspace), workspace.numel() * workspace.element_size(), ctypes.c_void_p(stream))
+    _check(rc)
+    return accepted_len, emitted_tokens, target_logits, draft_logits
+
+
+def from_hidden_status(workspace, B: int, n_draft_total: int, V: int, stream=None) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream(workspace.device).cuda_stream
+    return int(load().spec_verify_from_hidden_status(_ptr(workspace), B, n_draft_total, V, ctypes.c_void_p(stream)))

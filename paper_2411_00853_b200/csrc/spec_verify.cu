@@ -7,6 +7,7 @@
 #include <mutex>
 
 #include "specv_greedy_kernels.cuh"
+#include "specv_lmhead_kernel.cuh"
 #include "specv_ring_kernels.cuh"
 #include "specv_stream_kernels.cuh"
 #include "specv_tree_kernels.cuh"
@@ -31,6 +32,7 @@ struct DeviceInfo {
     int argmax_blocks_per_sm[3] = {0, 0, 0};
     int ring_argmax_ready[3] = {0, 0, 0};
     int tree_ready[3] = {0, 0, 0};
+    int lm_head_ready = 0;
 };
 DeviceInfo g_dev[kMaxDevices];
 std::mutex g_dev_mutex;   // guards the lazy per-device set-up (first call on a device from any thread)
@@ -984,4 +986,216 @@ extern "C" int spec_verify_debug_violation(void) {
 #else
     return -1;
 #endif
+}
+
+// ---------------------------------------------------------------------------------
+// spec_verify_from_hidden: LM-head products on the tensor cores with the row statistics in
+// their epilogue, then the resolve kernel of the ring set
+// ---------------------------------------------------------------------------------
+namespace {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn tensor_map_encoder() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// bf16 matrix [rows, cols] with a pitch of ld elements, boxes of box_rows x 64 elements, 128-byte swizzle
+bool make_bf16_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    EncodeTiledFn enc = tensor_map_encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)specv::kLmBK, (cuuint32_t)box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct HiddenLayout {
+    Workspace lay;
+    RingLayout rl;
+    size_t c_target, c_draft, part_t, part_d, status, total;
+};
+HiddenLayout hidden_layout(int32_t B, int64_t D, int64_t V) {
+    HiddenLayout h;
+    h.lay = workspace_layout(B, D, V);
+    h.rl = ring_layout(h.lay.total, B, D, V);
+    size_t o = h.rl.total;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    const size_t tiles_n = (size_t)((V + specv::kLmBN - 1) / specv::kLmBN);
+    h.c_target = take(sizeof(float) * (size_t)(D + B));
+    h.c_draft = take(sizeof(float) * (size_t)(D > 0 ? D : 1));
+    h.part_t = take(sizeof(float2) * (size_t)(D + B) * tiles_n);
+    h.part_d = take(sizeof(float2) * (size_t)(D > 0 ? D : 1) * tiles_n);
+    h.status = take(64);
+    h.total = o;
+    return h;
+}
+
+bool lm_head_ready(DeviceInfo& dev) {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (!dev.lm_head_ready) {
+        if (!cuda_ok(cudaFuncSetAttribute(specv::specv_lm_head, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)sizeof(specv::LmHeadShared))))
+            return false;
+        dev.lm_head_ready = 1;
+    }
+    return true;
+}
+
+int launch_lm_head(const void* hidden, int64_t ld_h, const void* weight, int64_t ld_w, int64_t M, int64_t V, int64_t H,
+                   const float* row_scale, void* logits, int64_t ld_out, float2* part, int32_t* status,
+                   DeviceInfo& dev, cudaStream_t stream) {
+    if (M == 0) return SPECV_OK;
+    CUtensorMap map_a, map_b;
+    if (!make_bf16_map(&map_a, hidden, M, H, ld_h, specv::kLmBM) || !make_bf16_map(&map_b, weight, V, H, ld_w, specv::kLmBN))
+        return SPECV_ERR_CUDA;
+    const int64_t tiles = ((M + specv::kLmBM - 1) / specv::kLmBM) * ((V + specv::kLmBN - 1) / specv::kLmBN);
+    const int grid = (int)(tiles < dev.sms ? tiles : dev.sms);
+    specv::specv_lm_head<<<grid, specv::kLmThreads, sizeof(specv::LmHeadShared), stream>>>(
+        map_a, map_b, M, V, H, row_scale, static_cast<uint16_t*>(logits), ld_out, part, status);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cuda_ok(cudaGetLastError()) ? SPECV_OK : SPECV_ERR_CUDA;
+}
+
+bool hidden_shape_ok(const void* hidden, int64_t ld_h, const void* weight, int64_t ld_w, int64_t H) {
+    // tensor maps: 16-byte aligned base addresses and pitches
+    return H >= 1 && ld_h >= H && ld_w >= H && !(reinterpret_cast<uintptr_t>(hidden) & 15u) &&
+           !(reinterpret_cast<uintptr_t>(weight) & 15u) && !((ld_h * 2) & 15) && !((ld_w * 2) & 15);
+}
+
+}  // namespace
+
+extern "C" size_t spec_verify_from_hidden_workspace_bytes(int32_t B, int64_t n_draft_total, int64_t V) {
+    if (!shape_ok(B, n_draft_total, V)) return 0;
+    return hidden_layout(B, n_draft_total, V).total;
+}
+
+extern "C" int spec_verify_from_hidden(const void* target_hidden, int64_t ld_th, int64_t H_target,
+                                       const void* target_weight, int64_t ld_tw, const void* draft_hidden,
+                                       int64_t ld_dh, int64_t H_draft, const void* draft_weight, int64_t ld_dw,
+                                       int64_t V, void* target_logits, int64_t ld_target, void* draft_logits,
+                                       int64_t ld_draft, const int32_t* draft_tokens, const int32_t* k_per_row,
+                                       int32_t B, int32_t k_uniform, int64_t n_draft_total, const float* temperature,
+                                       int temperature_per_row, const float* uniforms, int32_t* accepted_len,
+                                       int32_t* emitted_tokens, int32_t* row_status, float* diag_p_tok,
+                                       float* diag_q_tok, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    int rc = validate(target_logits, draft_logits, SPECV_BF16, V, ld_target, ld_draft, draft_tokens, k_per_row, B,
+                      k_uniform, n_draft_total, temperature, uniforms, accepted_len, emitted_tokens);
+    if (rc != SPECV_OK) return rc;
+    if (!target_hidden || !target_weight || !workspace) return SPECV_ERR_NULL;
+    if (n_draft_total > 0 && (!draft_hidden || !draft_weight)) return SPECV_ERR_NULL;
+    const int64_t D = n_draft_total;
+    if (!hidden_shape_ok(target_hidden, ld_th, target_weight, ld_tw, H_target)) return SPECV_ERR_SHAPE;
+    if (D > 0 && !hidden_shape_ok(draft_hidden, ld_dh, draft_weight, ld_dw, H_draft)) return SPECV_ERR_SHAPE;
+    if (!aligned_to(workspace, 256) || !aligned_to(draft_tokens, 4) || !aligned_to(k_per_row, 4) ||
+        !aligned_to(temperature, 4) || !aligned_to(uniforms, 4) || !aligned_to(accepted_len, 4) ||
+        !aligned_to(emitted_tokens, 4) || !aligned_to(row_status, 4) || !aligned_to(diag_p_tok, 4) ||
+        !aligned_to(diag_q_tok, 4))
+        return SPECV_ERR_ALIGN;
+    const HiddenLayout hl = hidden_layout(B, D, V);
+    if (workspace_bytes < hl.total) return SPECV_ERR_WORKSPACE;
+    DeviceInfo* dev = nullptr;
+    rc = device_info(&dev);
+    if (rc != SPECV_OK) return rc;
+
+    specv::BatchView in;
+    in.target = static_cast<const char*>(target_logits);
+    in.draft = static_cast<const char*>(draft_logits);
+    in.pitch_t = ld_target * 2;
+    in.pitch_d = ld_draft * 2;
+    in.V = V;
+    in.tokens = draft_tokens;
+    in.k_per_row = k_per_row;
+    in.B = B;
+    in.k_uniform = k_uniform;
+    in.n_draft_total = D;
+    in.temperature = temperature;
+    in.per_row_temperature = temperature_per_row ? 1 : 0;
+    in.uniforms = uniforms;
+    // the resolve kernel of the ring set reads the logits this call writes: their layout must be one it takes
+    if (!ring_shape_ok(in, SPECV_BF16)) return SPECV_ERR_SHAPE;
+    if (!ensure_ring_ready<specv::kBF16>(*dev) || !lm_head_ready(*dev)) return SPECV_ERR_CUDA;
+
+    char* ws = static_cast<char*>(workspace);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    using namespace specv;
+    RingScratch sc = {};
+    sc.off_d = reinterpret_cast<int32_t*>(ws + hl.lay.off_d);
+    sc.seq_status = reinterpret_cast<int32_t*>(ws + hl.lay.seq_status);
+    sc.stat_p = reinterpret_cast<float2*>(ws + hl.rl.stat_p);
+    sc.stat_q = reinterpret_cast<float2*>(ws + hl.rl.stat_q);
+    sc.done = reinterpret_cast<int32_t*>(ws + hl.rl.done);
+    sc.gseg = reinterpret_cast<float*>(ws + hl.rl.gseg);
+    sc.ctrl = reinterpret_cast<int32_t*>(ws + hl.rl.ctrl);
+    float* c_target = reinterpret_cast<float*>(ws + hl.c_target);
+    float* c_draft = reinterpret_cast<float*>(ws + hl.c_draft);
+    float2* part_t = reinterpret_cast<float2*>(ws + hl.part_t);
+    float2* part_d = reinterpret_cast<float2*>(ws + hl.part_d);
+    int32_t* lm_status = reinterpret_cast<int32_t*>(ws + hl.status);
+    g_last_path = 2;
+
+    // offsets, per-sequence checks, -1 fill, tickets and error word zeroed
+    const int64_t n_slots = D + B;
+    int pro_blocks = (int)((n_slots + 8 * kPrologueThreads - 1) / (8 * kPrologueThreads));
+    if (pro_blocks < 1) pro_blocks = 1;
+    if (pro_blocks > dev->sms) pro_blocks = dev->sms;
+    specv_prologue<<<pro_blocks, kPrologueThreads, 0, stream>>>(in, sc.off_d, sc.seq_status, emitted_tokens, sc.ctrl,
+                                                                  sc.done, 0);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (!cuda_ok(cudaGetLastError())) return SPECV_ERR_CUDA;
+    if (!cuda_ok(cudaMemsetAsync(lm_status, 0, 64, stream))) return SPECV_ERR_CUDA;
+    const int64_t n_rows = n_slots + D;
+    specv_row_scales<<<(unsigned)((n_rows + 255) / 256), 256, 0, stream>>>(in, sc.off_d, c_target, c_draft);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (!cuda_ok(cudaGetLastError())) return SPECV_ERR_CUDA;
+
+    rc = launch_lm_head(target_hidden, ld_th, target_weight, ld_tw, n_slots, V, H_target, c_target, target_logits,
+                        ld_target, part_t, lm_status, *dev, stream);
+    if (rc != SPECV_OK) return rc;
+    rc = launch_lm_head(draft_hidden, ld_dh, draft_weight, ld_dw, D, V, H_draft, c_draft, draft_logits, ld_draft, part_d,
+                        lm_status, *dev, stream);
+    if (rc != SPECV_OK) return rc;
+    const int64_t tiles_n = (V + kLmBN - 1) / kLmBN;
+    specv_merge_tile_stats<<<(unsigned)((n_slots * 32 + 255) / 256), 256, 0, stream>>>(part_t, n_slots, tiles_n, sc.stat_p);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (D > 0) {
+        specv_merge_tile_stats<<<(unsigned)((D * 32 + 255) / 256), 256, 0, stream>>>(part_d, D, tiles_n, sc.stat_q);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    if (!cuda_ok(cudaGetLastError())) return SPECV_ERR_CUDA;
+
+    const int64_t nck = (V * 2 + kChunkBytes - 1) / kChunkBytes;
+    const int64_t max_units = (int64_t)B * nck;
+    const int resolve_ctas = (int)(max_units < dev->sms ? max_units : dev->sms);
+    specv_ring_resolve<kBF16><<<resolve_ctas, kRingResolveThreads, sizeof(RingResolveShared), stream>>>(
+        in, sc, accepted_len, emitted_tokens, row_status, diag_p_tok, diag_q_tok, NextLookahead{nullptr, 0, 0});
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cuda_ok(cudaGetLastError()) ? SPECV_OK : SPECV_ERR_CUDA;
+}
+
+// Status word of the LM-head kernels of the last spec_verify_from_hidden call on this workspace
+// (0: no bounded wait expired).  Reads device memory: waits for the stream's work first.
+extern "C" int spec_verify_from_hidden_status(const void* workspace, int32_t B, int64_t n_draft_total, int64_t V,
+                                              void* cuda_stream) {
+    if (!workspace || !shape_ok(B, n_draft_total, V)) return -1;
+    const HiddenLayout hl = hidden_layout(B, n_draft_total, V);
+    int32_t v = 0;
+    if (!cuda_ok(cudaMemcpyAsync(&v, static_cast<const char*>(workspace) + hl.status, 4, cudaMemcpyDeviceToHost,
+                                 static_cast<cudaStream_t>(cuda_stream))) ||
+        !cuda_ok(cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream))))
+        return -2;
+    return v;
 }

@@ -313,3 +313,85 @@ def make_tree_config(*, B: int = 64, V: int = 128256, dtype: str = "bf16", seed:
               f"s_b ~ U[0.3,2.0]; T={temperature}")
     return TreeWorkload("tree", B, V, dtype, n, tl, dl, tok, T, uniforms, off_d, off_t, recipe,
                         node_parent=np.concatenate(parents).astype(np.int32), n_internal=int(sum(internal)))
+
+
+# ----------------------------------------------------------------------------- hidden states
+@dataclass
+class HiddenWorkload:
+    """Inputs of the verify pass one step earlier: hidden states and output-layer weights of both
+    models (bf16 bit patterns), from which the logits are a matrix product.  The draft tokens must be
+    drawn from the draft logits, which this module does not compute (no arithmetic of the method
+    here): the caller computes them with its own LM-head product and calls draw_tokens()."""
+    B: int
+    V: int
+    k_per_row: np.ndarray
+    target_hidden: np.ndarray     # uint16 [sum(K)+B, H]
+    target_weight: np.ndarray     # uint16 [V, H]
+    draft_hidden: np.ndarray      # uint16 [sum(K), Hd]
+    draft_weight: np.ndarray      # uint16 [V, Hd]
+    temperature: np.ndarray
+    uniforms: np.ndarray
+    off_d: np.ndarray
+    off_t: np.ndarray
+    seed: int
+
+    @property
+    def n_draft_total(self) -> int:
+        return int(self.off_d[-1])
+
+    def draw_tokens(self, draft_logits_bits: np.ndarray) -> np.ndarray:
+        """Draft tokens by Gumbel-max from softmax(draft logits / T) (bf16 bit patterns in)."""
+        tok = np.empty(self.n_draft_total, np.int32)
+        for b in range(self.B):
+            T = float(self.temperature[b] if self.temperature.shape[0] > 1 else self.temperature[0])
+            for i in range(int(self.k_per_row[b])):
+                g = _rng(self.seed, _STREAM_ROWS, (b << 8) | i)
+                e = g.standard_exponential(self.V, dtype=np.float32)
+                np.maximum(e, np.float32(1e-38), out=e)
+                row = bf16_bits_to_f32(draft_logits_bits[self.off_d[b] + i])
+                tok[self.off_d[b] + i] = int(np.argmax(row / np.float32(T) - np.log(e)))
+        return tok
+
+
+def make_hidden_config(*, B: int, V: int, H: int, Hd: int | None = None, K: int | None = None, seed: int = 6,
+                       exact: bool = True, temperature: float = 0.8) -> HiddenWorkload:
+    """Seeded hidden states and weights.  exact=True: every product and every sum of the matrix
+    product is exactly representable -- hidden states with 24 non-zero entries per row from
+    {+-1/4, +-1/2}, weights integers in [-2, 2] -- so the logits are multiples of 1/4 below 32 in
+    magnitude, which bf16 holds exactly, and any correct product gives the same bytes whatever its
+    accumulation order.  The draft model's hidden state is the target's with a third of the non-zero
+    entries redrawn (so the two models mostly agree); exact=False: N(0,1) hidden states and
+    N(0, 1/H) weights (no exactness; for timing).  K: fixed lookahead, else ragged 1..8."""
+    Hd = H if Hd is None else Hd
+    g = _rng(seed, _STREAM_SCALARS, 0)
+    k = np.full(B, K, np.int32) if K is not None else g.integers(1, 9, size=B).astype(np.int32)
+    off_d = np.concatenate([[0], np.cumsum(k)]).astype(np.int64)
+    off_t = off_d[:-1] + np.arange(B)
+    D = int(off_d[-1])
+    if exact:
+        def sparse_rows(n, width, gen):
+            a = np.zeros((n, width), np.float32)
+            for r in range(n):
+                idx = gen.choice(width, size=min(24, width), replace=False)
+                a[r, idx] = gen.choice(np.array([-0.5, -0.25, 0.25, 0.5], np.float32), size=idx.size)
+            return a
+        th = sparse_rows(D + B, H, g)
+        dh = np.zeros((D, Hd), np.float32)
+        for b in range(B):
+            for i in range(int(k[b])):
+                row = th[off_t[b] + i, :min(H, Hd)].copy()
+                nz = np.nonzero(row)[0]
+                redo = nz[g.random(nz.size) < 1.0 / 3.0]
+                row[redo] = g.choice(np.array([-0.5, -0.25, 0.25, 0.5], np.float32), size=redo.size)
+                dh[off_d[b] + i, :row.size] = row
+        tw = g.integers(-2, 3, size=(V, H)).astype(np.float32)
+        dw = tw[:, :Hd].copy() if Hd <= H else np.concatenate([tw, g.integers(-2, 3, size=(V, Hd - H)).astype(np.float32)], 1)
+    else:
+        th = g.standard_normal((D + B, H), dtype=np.float32)
+        dh = g.standard_normal((D, Hd), dtype=np.float32)
+        tw = g.standard_normal((V, H), dtype=np.float32) * np.float32(3.0 / np.sqrt(H))
+        dw = g.standard_normal((V, Hd), dtype=np.float32) * np.float32(3.0 / np.sqrt(Hd))
+    gu = _rng(seed, _STREAM_UNIFORMS, 0)
+    uniforms = gu.integers(0, 1 << 24, size=D + B).astype(np.float32) * np.float32(2.0 ** -24)
+    return HiddenWorkload(B, V, k, f32_to_bf16_bits(th), f32_to_bf16_bits(tw), f32_to_bf16_bits(dh), f32_to_bf16_bits(dw),
+                          np.array([temperature], np.float32), uniforms, off_d, off_t, seed)
