@@ -597,6 +597,8 @@ TreeLayout tree_layout(int32_t B, int64_t D, int64_t V) {
     return t;
 }
 
+constexpr int kTreeMaxSmem = 200 * 1024;     // caches (52 KB) and the segment sums of the largest vocabulary (128 KB)
+
 template <int DT>
 int launch_tree(specv::BatchView in, const TreeLayout& tl, char* ws, DeviceInfo& dev, bool ring,
                 int32_t* accepted_len, int32_t* emitted, int32_t* accepted_nodes, int32_t* row_status,
@@ -613,8 +615,8 @@ int launch_tree(specv::BatchView in, const TreeLayout& tl, char* ws, DeviceInfo&
     {
     std::lock_guard<std::mutex> lock(g_dev_mutex);
     if (!dev.tree_ready[DT]) {
-        if (!cuda_ok(cudaFuncSetAttribute(specv_tree_resolve<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          160 * 1024)))
+        if (!cuda_ok(cudaFuncSetAttribute(specv_tree_resolve<DT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTreeMaxSmem)) ||
+            !cuda_ok(cudaFuncSetAttribute(specv_tree_resolve<DT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTreeMaxSmem)))
             return SPECV_ERR_CUDA;
         dev.tree_ready[DT] = 1;
     }
@@ -679,14 +681,30 @@ int launch_tree(specv::BatchView in, const TreeLayout& tl, char* ws, DeviceInfo&
 
     trace(2);
     const int seg_elems = 32 * Elt<DT>::kPerVec;
-    cfg.gridDim = dim3((unsigned)in.B, 1, 1);
+    const size_t nseg = (size_t)((in.V + seg_elems - 1) / seg_elems);
+    // pairs of CTAs per sequence while every pair still gets SMs of its own: a walk is a chain of
+    // dependent passes, and a pair halves the time of each
+    const size_t seg_bytes = sizeof(float) * ((nseg + 3) & ~(size_t)3);
+    const bool pairs = 2 * (int64_t)in.B <= dev.sms && kTreeCacheBytes + 2 * seg_bytes <= (size_t)kTreeMaxSmem;
+    cudaLaunchAttribute attrs[2];
+    attrs[0] = pdl[0];
+    attrs[1].id = cudaLaunchAttributeClusterDimension;
+    attrs[1].val.clusterDim.x = 2;
+    attrs[1].val.clusterDim.y = 1;
+    attrs[1].val.clusterDim.z = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = pairs ? 2 : 1;
+    cfg.gridDim = dim3((unsigned)in.B * (pairs ? 2u : 1u), 1, 1);
     cfg.blockDim = dim3(kTreeThreads, 1, 1);
-    cfg.dynamicSmemBytes = sizeof(float) * (size_t)((in.V + seg_elems - 1) / seg_elems);
+    cfg.dynamicSmemBytes = kTreeCacheBytes + (pairs ? 2 : 1) * seg_bytes;      // a pair alternates between two buffers
     const int32_t* seq_status_c = seq_status;
     const int32_t* err_c = ring ? ctrl : nullptr;
-    if (!cuda_ok(cudaLaunchKernelEx(&cfg, specv_tree_resolve<DT>, in, off_d_c, seq_status_c, stat_t, stat_d, splits,
-                                    err_c, accepted_len, emitted, accepted_nodes, row_status, diag_p, diag_q)))
-        return SPECV_ERR_CUDA;
+    const cudaError_t e =
+        pairs ? cudaLaunchKernelEx(&cfg, specv_tree_resolve<DT, 2>, in, off_d_c, seq_status_c, stat_t, stat_d, splits, err_c,
+                                   accepted_len, emitted, accepted_nodes, row_status, diag_p, diag_q)
+              : cudaLaunchKernelEx(&cfg, specv_tree_resolve<DT, 1>, in, off_d_c, seq_status_c, stat_t, stat_d, splits, err_c,
+                                   accepted_len, emitted, accepted_nodes, row_status, diag_p, diag_q);
+    if (!cuda_ok(e)) return SPECV_ERR_CUDA;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     trace(3);
     return SPECV_OK;

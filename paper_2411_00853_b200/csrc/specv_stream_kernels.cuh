@@ -377,8 +377,9 @@ __device__ int32_t locate_in_segments(const SampleRows& sr, int64_t V, double u,
 // segment); NWARPS warps take part, `warp` in [0, NWARPS) being the caller's index among them;
 // `sync` is a barrier over exactly those warps and is called once at the end.
 // FAST: both rows start on 16-byte boundaries and V is a whole number of vectors.
-template <int DT, int NWARPS, bool FAST, class SyncFn>
-__device__ void block_segment_sums(const SampleRows& sr, int64_t V, float* seg, int warp, SyncFn sync) {
+// `store(s, a)` receives the mass a of segment s from lane 0 of the warp that summed it.
+template <int DT, int NWARPS, bool FAST, class StoreFn, class SyncFn>
+__device__ void block_segment_sums_to(const SampleRows& sr, int64_t V, int warp, StoreFn store, SyncFn sync) {
     using E = Elt<DT>;
     constexpr int N = E::kPerVec;
     constexpr int SEG = 32 * N;                 // elements per warp-wide segment
@@ -412,11 +413,15 @@ __device__ void block_segment_sums(const SampleRows& sr, int64_t V, float* seg, 
 #pragma unroll
                 for (int k = 0; k < N; ++k) a += r[k];
                 a = warp_sum(a);
-                if (lane == 0) seg[s] = a;
+                if (lane == 0) store(s, a);
             }
         }
     }
     sync();
+}
+template <int DT, int NWARPS, bool FAST, class SyncFn>
+__device__ void block_segment_sums(const SampleRows& sr, int64_t V, float* seg, int warp, SyncFn sync) {
+    block_segment_sums_to<DT, NWARPS, FAST>(sr, V, warp, [seg](int32_t s, float a) { seg[s] = a; }, sync);
 }
 
 // Total of the segment masses, summed in double exactly as locate_in_segments sums them (a
