@@ -390,25 +390,30 @@ __device__ void block_segment_sums_to(const SampleRows& sr, int64_t V, int warp,
         return load_vec<DT>(row, aligned, v, V);
     };
     // segments dealt round-robin to warps (vocabulary order kept by the segment index, so the
-    // prefix taken later is over token ids); four segments per warp and iteration, all loads
-    // issued before any arithmetic
-    constexpr int U = 4;
-    for (int32_t s0 = warp; s0 < nseg; s0 += U * NWARPS) {
-        uint4 rawp[U], rawq[U];
+    // prefix taken later is over token ids); two segments per warp and step, and the loads of the
+    // next step are issued before the arithmetic of this one (the exponentials of a step take as
+    // long as its loads, so neither waits for the other)
+    constexpr int U = 2;
+    uint4 curp[U], curq[U], nxtp[U], nxtq[U];
+    auto issue = [&](int32_t s0, uint4* rp, uint4* rq) {
 #pragma unroll
         for (int i = 0; i < U; ++i) {
             const int32_t s = s0 + i * NWARPS;
             if (s < nseg) {
-                rawp[i] = load(sr.p, sr.p_aligned, (int64_t)s * 32 + lane);
-                rawq[i] = sr.q ? load(sr.q, sr.q_aligned, (int64_t)s * 32 + lane) : make_uint4(0u, 0u, 0u, 0u);
+                rp[i] = load(sr.p, sr.p_aligned, (int64_t)s * 32 + lane);
+                rq[i] = sr.q ? load(sr.q, sr.q_aligned, (int64_t)s * 32 + lane) : make_uint4(0u, 0u, 0u, 0u);
             }
         }
+    };
+    if (warp < nseg) issue(warp, curp, curq);
+    for (int32_t s0 = warp; s0 < nseg; s0 += U * NWARPS) {
+        if (s0 + U * NWARPS < nseg) issue(s0 + U * NWARPS, nxtp, nxtq);
 #pragma unroll
         for (int i = 0; i < U; ++i) {
             const int32_t s = s0 + i * NWARPS;
             if (s < nseg) {      // warp-uniform
                 float r[N];
-                mass_of_raw<DT>(sr, rawp[i], rawq[i], r);
+                mass_of_raw<DT>(sr, curp[i], curq[i], r);
                 float a = 0.f;
 #pragma unroll
                 for (int k = 0; k < N; ++k) a += r[k];
@@ -416,6 +421,8 @@ __device__ void block_segment_sums_to(const SampleRows& sr, int64_t V, int warp,
                 if (lane == 0) store(s, a);
             }
         }
+#pragma unroll
+        for (int i = 0; i < U; ++i) { curp[i] = nxtp[i]; curq[i] = nxtq[i]; }
     }
     sync();
 }
