@@ -109,6 +109,22 @@ def test_small_and_odd_vocabularies(dtype, V):
         assert ora.accepted_len.max() >= 2
 
 
+def test_one_cta_and_paired_ctas_give_the_same_walks():
+    """A batch of at most half as many sequences as the device has SMs is resolved by a pair of CTAs
+    per sequence, a larger one by single CTAs: the first 60 sequences of a batch of 100 (single CTAs) must
+    come out exactly as when they are submitted alone (pairs), and both must agree with the oracle."""
+    w = W.make_tree_config(B=100, V=6001, dtype="bf16", seed=21)
+    got_all = run_gpu(w)
+    acc_all, em_all, nodes_all = got_all[:3]
+    assert_tree_parity(w, got_all, max_excused_frac=0.05)
+    sub = w.take(0, 60)
+    acc, em, nodes = run_gpu(sub)[:3]
+    n_slots = sub.n_draft_total + sub.B
+    assert np.array_equal(acc, acc_all[:60])
+    assert np.array_equal(em[:n_slots], em_all[:n_slots])
+    assert np.array_equal(nodes[:n_slots], nodes_all[:n_slots])
+
+
 def test_many_siblings():
     """A root with twelve children drawn from a poor draft: long runs of rejections, each with its
     own pass and coefficient."""
