@@ -35,8 +35,8 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
 # kernel from the ncu capture summarised under profiles/; only valid for the kernel source
 # it was taken from (sha256 of the files that kernel is compiled from), otherwise reported as null.
-NCU_TRAFFIC = {"csrc_sha256": "07238c5e9337cac0d2f6be18a5449e07ec693a84105dc7fa9299e8e37fc82a17",
-               "workload": "config3 capture of specv_ring_stats scaled by rows to config5", "bytes_per_launch": 2434715520}
+NCU_TRAFFIC = {"csrc_sha256": "b39e20532d800f3a2bfe461818343381e018b694d731356f3c6fe4dc3127ceea",
+               "workload": "config3 capture of specv_ring_stats (279.14 MB read + 4.20 MB written for 279.09 MB of logits) scaled by logit bytes to config5", "bytes_per_launch": 2425103345}
 
 
 # the sources the dominant kernel (specv_ring_stats) is compiled from
