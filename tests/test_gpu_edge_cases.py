@@ -115,3 +115,24 @@ def test_second_uniform_of_exactly_one(kernel_path, cfg, B, V):
         assert em[m.off_t[b] + acc[b]] in kept[b]
         if acc[b] == m.k_per_row[b]:                    # bonus draw: the last kept id has mass under p
             assert em[m.off_t[b] + acc[b]] >= kept[b][-1] - 512      # within the last segment that has mass
+
+
+@pytest.mark.parametrize("cfg", [1, 2])      # fp32 and bf16 logits
+def test_largest_vocabulary(kernel_path, cfg):
+    """The largest vocabulary the library takes (2^22 entries: the segment table of the sampler is
+    then at its shared-memory limit), two sequences: parity as usual; one entry more is refused."""
+    V = 1 << 22
+    w = W.make_config(cfg, B=2, V=V, K=2)
+    got = DeviceBatch(w).run()
+    assert_parity(w, got, max_excused_frac=0.5)
+    assert binding.workspace_bytes(2, 4, V) > 0
+    assert binding.workspace_bytes(2, 4, V + 1) == 0
+
+
+def test_largest_vocabulary_tree():
+    """Tree walk at 2^22 entries: fp32 logits (one CTA per sequence: two segment tables would not
+    fit) and bf16 logits (pairs of CTAs)."""
+    import test_gpu_tree as T
+    for dtype in ("f32", "bf16"):
+        w = W.make_tree_config(B=2, V=1 << 22, dtype=dtype, seed=31, depth=2, max_level_width=3)
+        T.assert_tree_parity(w, T.run_gpu(w), max_excused_frac=0.5)

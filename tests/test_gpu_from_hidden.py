@@ -32,7 +32,9 @@ def _oracle_side(w):
 @pytest.mark.parametrize("B,V,H,Hd,K", [(6, 512, 64, 64, 2),          # one column tile pair, one k-block
                                          (20, 4096, 256, 128, None),   # several k-blocks, ragged lookahead
                                          (37, 20000, 320, 192, None),  # ragged last column tile, ragged last row tile, H not a multiple of 64
-                                         (150, 2048, 128, 128, 3)])    # many row tiles
+                                         (150, 2048, 128, 128, 3),     # many row tiles
+                                         (32, 256, 64, 64, 3),         # exactly one 128 x 256 tile of target logits
+                                         (43, 264, 192, 64, 2)])       # 129 target rows; 8 columns past a column tile
 def test_logits_are_exact_and_the_pass_matches_the_oracle(B, V, H, Hd, K):
     w = W.make_hidden_config(B=B, V=V, H=H, Hd=Hd, K=K)
     tl, dl, tok, case, ora = _oracle_side(w)
