@@ -136,3 +136,13 @@ def test_largest_vocabulary_tree():
     for dtype in ("f32", "bf16"):
         w = W.make_tree_config(B=2, V=1 << 22, dtype=dtype, seed=31, depth=2, max_level_width=3)
         T.assert_tree_parity(w, T.run_gpu(w), max_excused_frac=0.5)
+
+
+@pytest.mark.parametrize("B", [4095, 4096, 6000])
+def test_batch_sizes_around_the_ring_kernels_limit(kernel_path, B):
+    """The ring kernels keep one offset per sequence in shared memory and take up to 4095 sequences; a
+    larger batch goes to the streaming kernels whatever the call asks for."""
+    w = W.make_config(5, B=B, V=1024)
+    got = DeviceBatch(w).run()
+    _expect_path(kernel_path, ring_capable=B <= 4095)
+    assert_parity(w, got, max_excused_frac=0.02)
