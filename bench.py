@@ -39,6 +39,10 @@ NCU_TRAFFIC = {"csrc_sha256": "b39e20532d800f3a2bfe461818343381e018b694d731356f3
                "workload": "config3 capture of specv_ring_stats (279.14 MB read + 4.20 MB written for 279.09 MB of logits) scaled by logit bytes to config5", "bytes_per_launch": 2425103345}
 
 
+# kernel set of a pass as spec_verify_last_path reports it
+PATH_NAMES = {1: "streaming", 2: "ring", 3: "cluster"}
+
+
 # the sources the dominant kernel (specv_ring_stats) is compiled from
 DOMINANT_KERNEL_SOURCES = ("specv_device.cuh", "specv_stream_kernels.cuh", "specv_ring_kernels.cuh")
 
@@ -402,7 +406,7 @@ def greedy_leg(dw, w, device, steps, warmup, flush, peak):
     return {"ms_per_step": ms, "value": w.n_draft_total / (ms * 1e-3), "unit": UNIT,
             "bytes_per_pass": int(rows * row_bytes), "argmax_kernel_ms": k_ms[1], "argmax_kernel_gbs": gbs,
             "argmax_kernel_frac": gbs / peak, "whole_pass_frac": rows * row_bytes / (ms * 1e-3) / 1e9 / peak,
-            "path": {1: "streaming", 2: "ring"}[dw.binding.last_path()],
+            "path": PATH_NAMES[dw.binding.last_path()],
             "parity_sample": {"sequences": n_seq, "exact": exact},
             "note": "temperature -> 0 limit: accept while the draft token is the target argmax; target rows only"}
 
@@ -440,7 +444,7 @@ def tree_leg(device, steps, warmup, peak):
         ora.emitted_tokens[int(sub.off_t[b]):int(sub.off_t[b]) + int(sub.k_per_row[b]) + 1]) for b in range(n_seq)))
     return {"ms_per_step": ms, "nodes": int(D), "sequences": int(B), "value": D / (ms * 1e-3), "unit": "tree nodes/s",
             "bytes_first_pass": int(w.logit_bytes), "first_pass_frac_of_peak": w.logit_bytes / (ms * 1e-3) / 1e9 / peak,
-            "path": {1: "streaming", 2: "ring"}[binding.last_path()],
+            "path": PATH_NAMES[binding.last_path()],
             "parity_sample": {"sequences": n_seq, "identical": same},
             "note": "every rejected sibling costs one more pass over its context's two rows, so the pass reads "
                     "more than bytes_first_pass; the fraction is a lower bound on the achieved bandwidth"}
@@ -581,11 +585,12 @@ def run_ours(args):
     positions = w.n_draft_total * world
     peak, peak_kind = measured_peak_gbs()
     stats_ms = k_ms[1]
-    ring = binding.last_path() >= 2
+    ring = binding.last_path() == 2
     # the ring kernel set has no prologue kernel (its statistics kernel does that work): the
     # first interval is then only the gap between two event records
     names = {1: ["specv_prologue", "specv_row_stats", "specv_resolve"],
-             2: ["(event gap)", "specv_ring_stats", "specv_ring_resolve"]}[binding.last_path()]
+             2: ["(event gap)", "specv_ring_stats", "specv_ring_resolve"],
+             3: ["(event gap)", "specv_cluster_pass", "(event gap after)"]}[binding.last_path()]
     traffic = (NCU_TRAFFIC["bytes_per_launch"]
                if ring and args.config == 5 and NCU_TRAFFIC["csrc_sha256"] == csrc_sha256() else None)
     achieved = w.logit_bytes / (stats_ms * 1e-3) / 1e9
@@ -726,7 +731,7 @@ def run_ours(args):
                                 "input_sets": input_sets(wc),
                                 "k_per_row": "NULL (uniform lookahead)" if dw.k_uniform is not None else "device array",
                                 "graph_replay_us_no_flush": graph_replay_us(dw),
-                                "path": {1: "streaming", 2: "ring"}[binding.last_path()]}
+                                "path": PATH_NAMES[binding.last_path()]}
             line["all_configs"] = allc
     if rank == 0:
         print(json.dumps(line), flush=True)

@@ -73,7 +73,16 @@ enum {
                                    else streaming.  Neither bit: automatic, the ring kernels from 64
                                    target rows up.  Results of the two sets agree except for draws within
                                    rounding of a decision boundary. */
-    SPECV_FLAG_EARLY_EXIT = 4   /* spec_verify_ex only; see there */
+    SPECV_FLAG_EARLY_EXIT = 4,  /* spec_verify_ex only; see there */
+    SPECV_FLAG_CLUSTER = 8      /* the one-launch form for small batches: a thread-block cluster of eight
+                                   CTAs per sequence keeps all of the sequence's logits rows in shared
+                                   memory (every logit fetched once, no workspace traffic).  Taken when
+                                   the batch has at most 18 sequences, rows on 16-byte boundaries with
+                                   V*elt a multiple of 16, a lookahead of at most 32 (if k_per_row is
+                                   given the host cannot see it and n_draft_total must be at most 32),
+                                   and (2K+1) rows of ceil(V*elt/512/8)*512 bytes fit in 200 KB; else
+                                   the automatic choice.  The automatic choice (no kernel-set bit)
+                                   takes this form whenever those conditions hold. */
 };
 
 /* Bits of row_status[b] (data errors found on the device; the call itself succeeds).
@@ -157,7 +166,7 @@ int spec_verify(const void* target_logits, const void* draft_logits, int dtype,
  * spec_verify with per-call options and, optionally, the lookahead of the next speculation round
  * written by the same kernels.  spec_verify(...) is spec_verify_ex(..., 0, 0, 0, NULL).
  *
- *   flags   SPECV_FLAG_STREAMING or SPECV_FLAG_RING (kernel set; neither: automatic), and
+ *   flags   SPECV_FLAG_STREAMING, SPECV_FLAG_RING or SPECV_FLAG_CLUSTER (kernel set; none: automatic), and
  *           SPECV_FLAG_EARLY_EXIT: the paper's theme is to do only the work the input needs; in this
  *           pass nothing after a sequence's first rejected draft token can be emitted, so the logits
  *           rows of later positions need not be read.  With this flag the ring kernels process the
@@ -186,7 +195,7 @@ int spec_verify_ex(const void* target_logits, const void* draft_logits, int dtyp
                    uint32_t flags, int32_t k_min, int32_t k_max, int32_t* next_k);
 
 /* Kernel set the calling thread's most recent pass (any entry point below or above) used:
- * 1 streaming, 2 ring, 0 if it has made none.  Not a status code. */
+ * 1 streaming, 2 ring, 3 the one-launch cluster form, 0 if it has made none.  Not a status code. */
 int spec_verify_last_path(void);
 
 /*

@@ -125,8 +125,9 @@ def set_trace_events(events):
     lib.spec_verify_set_trace_events(arr)
 
 
-PATH_AUTO, PATH_STREAMING, PATH_RING = 0, 1, 2
-FLAG_STREAMING, FLAG_RING, FLAG_EARLY_EXIT = 1, 2, 4
+PATH_AUTO, PATH_STREAMING, PATH_RING, PATH_CLUSTER = 0, 1, 2, 3
+FLAG_STREAMING, FLAG_RING, FLAG_EARLY_EXIT, FLAG_CLUSTER = 1, 2, 4, 8
+_PATH_FLAG = {PATH_AUTO: 0, PATH_STREAMING: FLAG_STREAMING, PATH_RING: FLAG_RING, PATH_CLUSTER: FLAG_CLUSTER}
 
 # The C library keeps no mode between calls: options travel with every call as `flags`.  For
 # convenience (tests, the benchmark) this module holds DEFAULT flags that its wrappers pass when
@@ -135,11 +136,11 @@ _default_flags = 0
 
 
 def set_path(path: int):
-    """Default kernel set of this module's wrappers: PATH_AUTO, PATH_STREAMING or PATH_RING."""
+    """Default kernel set of this module's wrappers: PATH_AUTO, PATH_STREAMING, PATH_RING or PATH_CLUSTER."""
     global _default_flags
-    if path not in (PATH_AUTO, PATH_STREAMING, PATH_RING):
-        raise ValueError("path must be PATH_AUTO, PATH_STREAMING or PATH_RING")
-    _default_flags = (_default_flags & ~(FLAG_STREAMING | FLAG_RING)) | path
+    if path not in _PATH_FLAG:
+        raise ValueError("path must be PATH_AUTO, PATH_STREAMING, PATH_RING or PATH_CLUSTER")
+    _default_flags = (_default_flags & ~(FLAG_STREAMING | FLAG_RING | FLAG_CLUSTER)) | _PATH_FLAG[path]
 
 
 def set_early_exit(enable: bool):

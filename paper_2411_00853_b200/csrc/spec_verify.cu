@@ -6,6 +6,7 @@
 #include <cstring>
 #include <mutex>
 
+#include "specv_cluster_kernels.cuh"
 #include "specv_greedy_kernels.cuh"
 #include "specv_lmhead_kernel.cuh"
 #include "specv_ring_kernels.cuh"
@@ -33,6 +34,7 @@ struct DeviceInfo {
     int ring_argmax_ready[3] = {0, 0, 0};
     int tree_ready[3] = {0, 0, 0};
     int lm_head_ready = 0;
+    int cluster_ready[3] = {0, 0, 0};
 };
 DeviceInfo g_dev[kMaxDevices];
 std::mutex g_dev_mutex;   // guards the lazy per-device set-up (first call on a device from any thread)
@@ -379,9 +381,64 @@ int spec_verify_last_path(void) { return g_last_path; }
 
 namespace {
 
-constexpr uint32_t kKnownFlags = SPECV_FLAG_STREAMING | SPECV_FLAG_RING | SPECV_FLAG_EARLY_EXIT;
+constexpr uint32_t kKnownFlags = SPECV_FLAG_STREAMING | SPECV_FLAG_RING | SPECV_FLAG_EARLY_EXIT | SPECV_FLAG_CLUSTER;
 bool flags_ok(uint32_t flags) {
-    return !(flags & ~kKnownFlags) && (flags & (SPECV_FLAG_STREAMING | SPECV_FLAG_RING)) != (SPECV_FLAG_STREAMING | SPECV_FLAG_RING);
+    const uint32_t set = flags & (SPECV_FLAG_STREAMING | SPECV_FLAG_RING | SPECV_FLAG_CLUSTER);
+    return !(flags & ~kKnownFlags) && !(set & (set - 1));       // at most one kernel set
+}
+
+// The one-launch form for small batches (specv_cluster_kernels.cuh): a cluster of eight CTAs per
+// sequence must hold every row of the sequence in shared memory.  The host knows the lookahead only
+// when it is uniform; for a ragged batch the number of draft rows bounds it.
+constexpr size_t kClusterSmemLimit = 200 * 1024;
+struct ClusterPlan {
+    bool ok = false;
+    int32_t slice_bytes = 0;
+    size_t smem = 0;
+};
+ClusterPlan cluster_plan(const specv::BatchView& in, int dtype, uint32_t flags) {
+    ClusterPlan p;
+    if (flags & (SPECV_FLAG_STREAMING | SPECV_FLAG_RING | SPECV_FLAG_EARLY_EXIT)) return p;
+    const int64_t elt = dtype == SPECV_F32 ? 4 : 2;
+    if (in.B > specv::kClusterMaxSeqs) return p;
+    if ((reinterpret_cast<uintptr_t>(in.target) & 15u) || (in.pitch_t & 15) || ((in.V * elt) & 15)) return p;
+    if (in.n_draft_total > 0 && ((reinterpret_cast<uintptr_t>(in.draft) & 15u) || (in.pitch_d & 15))) return p;
+    const int64_t k_bound = in.k_per_row ? in.n_draft_total : (in.k_uniform > 0 ? in.k_uniform : 0);
+    if (k_bound > specv::kClusterMaxK) return p;
+    const int64_t row_bytes = in.V * elt;
+    const int64_t nseg = (row_bytes + 511) / 512;
+    const int64_t slice = ((nseg + specv::kClusterCtas - 1) / specv::kClusterCtas) * 512;
+    const size_t smem = (size_t)(2 * k_bound + 1) * (size_t)slice + sizeof(float) * (size_t)nseg;
+    if (smem > kClusterSmemLimit) return p;
+    p.ok = true;
+    p.slice_bytes = (int32_t)slice;
+    p.smem = smem;
+    return p;
+}
+
+template <int DT>
+int launch_cluster_path(const specv::BatchView& in, const ClusterPlan& plan, DeviceInfo& dev, int32_t* accepted_len,
+                        int32_t* emitted, int32_t* row_status, float* diag_p, float* diag_q, specv::NextLookahead next,
+                        cudaStream_t stream) {
+    using namespace specv;
+    {
+        std::lock_guard<std::mutex> lock(g_dev_mutex);
+        if (!dev.cluster_ready[DT]) {
+            if (!cuda_ok(cudaFuncSetAttribute(specv_cluster_pass<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kClusterSmemLimit)))
+                return SPECV_ERR_CUDA;
+            dev.cluster_ready[DT] = 1;
+        }
+    }
+    auto trace = [&](int i) { if (g_trace_on) cudaEventRecord(g_trace[i], stream); };
+    trace(0);
+    trace(1);
+    specv_cluster_pass<DT><<<in.B * kClusterCtas, kClusterThreads, plan.smem, stream>>>(
+        in, plan.slice_bytes, accepted_len, emitted, row_status, diag_p, diag_q, next);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    trace(2);
+    trace(3);
+    return cuda_ok(cudaGetLastError()) ? SPECV_OK : SPECV_ERR_CUDA;
 }
 // Kernel set for a batch of n_items work items whose shape the ring kernels can (or cannot) take.
 // They give a whole (target row, draft row) item to one CTA, so they need enough items to occupy
@@ -428,6 +485,20 @@ int run_pass(const void* target_logits, const void* draft_logits, int dtype, int
     const specv::NextLookahead next{next_k, k_min, k_max};
     const bool early = (flags & SPECV_FLAG_EARLY_EXIT) != 0;
 
+    // small batches: everything in one launch, if a cluster per sequence can hold the sequence's rows
+    // and the device runs that many clusters at once
+    const ClusterPlan cluster = cluster_plan(in, dtype, flags);
+    if (cluster.ok && B * specv::kClusterCtas <= dev->sms) {
+        g_last_path = 3;
+        if (dtype == SPECV_F32)
+            return launch_cluster_path<specv::kF32>(in, cluster, *dev, accepted_len, emitted_tokens, row_status,
+                                                    diag_p_tok, diag_q_tok, next, stream);
+        if (dtype == SPECV_F16)
+            return launch_cluster_path<specv::kF16>(in, cluster, *dev, accepted_len, emitted_tokens, row_status,
+                                                    diag_p_tok, diag_q_tok, next, stream);
+        return launch_cluster_path<specv::kBF16>(in, cluster, *dev, accepted_len, emitted_tokens, row_status,
+                                                 diag_p_tok, diag_q_tok, next, stream);
+    }
     if (choose_ring(flags, ring_shape_ok(in, dtype), n_draft_total + B)) {
         g_last_path = 2;
         if (dtype == SPECV_F32)

@@ -1,0 +1,311 @@
+// The whole pass in ONE launch for small batches (one to a dozen sequences): a thread-block cluster
+// of eight CTAs per sequence holds every logits row of the sequence in its shared memory.
+//
+// For a handful of sequences the pass is not bound by HBM but by latency: three dependent launches
+// (offsets, row statistics, resolve), each with its own round of loads, and a second read of the
+// row pair a token is drawn from.  Here every logit is fetched exactly once:
+//   CTA r of a cluster takes the columns [r, r+1) * slice of EVERY row of its sequence (K+1 target
+//   rows, K draft rows) with bulk async copies into shared memory (all in flight at once);
+//   one warp per row computes the (reference, sum) of its slice and writes it into the partials
+//   table of all eight CTAs through distributed shared memory; after one cluster barrier every CTA
+//   holds the statistics of every row and takes the decisions (all positions in parallel, in
+//   double, first rejection) redundantly and identically;
+//   the segment sums of the distribution the token is drawn from are computed from the slices
+//   still in shared memory and written to the segment table of all eight CTAs; after a second
+//   cluster barrier CTA 0 locates the token (prefix over the table, one 512-byte segment re-read
+//   from L2) and writes the sequence's outputs.
+// No workspace, no atomics in global memory, no wait on another CTA other than the hardware cluster
+// barrier; the one bounded wait is for the CTA's own copies.
+//
+// Same arithmetic as the streaming kernels: statistics merged per row in double in a fixed order
+// (warp_merge_splits over the eight partials), decisions u q < p in double, masses by mass_of_raw,
+// inverse CDF by locate_in_segments.
+#pragma once
+
+#include "specv_ring_kernels.cuh"
+
+namespace specv {
+
+constexpr int kClusterCtas = 8;
+constexpr int kClusterThreads = 512;
+constexpr int kClusterWarps = kClusterThreads / 32;
+constexpr int kClusterMaxK = 32;                          // lookahead the shared-memory tables are sized for
+constexpr int kClusterMaxRows = 2 * kClusterMaxK + 1;
+constexpr int kClusterMaxSeqs = 18;                       // 8 CTAs each on 148 SMs; offsets are scanned by one warp
+
+struct ClusterShared {
+    float2 part[kClusterMaxRows * kClusterCtas];          // [row][cta]: partial (ref, sum) of every row from every CTA
+    int err_of[kClusterCtas];                             // a CTA whose copies did not arrive reports here, everywhere
+    unsigned long long bar;
+    SampleRows rows;
+    int32_t first_reject, bad_token, err;
+};
+
+__device__ __forceinline__ uint32_t map_to_cta(const void* smem_ptr, uint32_t cta) {
+    uint32_t a;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(smem_u32(smem_ptr)), "r"(cta));
+    return a;
+}
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Dynamic shared memory: the slices of the sequence's rows (row-major, `slice_bytes` each, 16-byte
+// aligned), then the segment table (one float per 512-byte segment of a row).
+template <int DT>
+__global__ void __cluster_dims__(kClusterCtas, 1, 1) __launch_bounds__(kClusterThreads, 1)
+specv_cluster_pass(BatchView in, int32_t slice_bytes, int32_t* __restrict__ accepted_len, int32_t* __restrict__ emitted,
+                   int32_t* __restrict__ row_status, float* __restrict__ diag_p, float* __restrict__ diag_q,
+                   NextLookahead next) {
+    using E = Elt<DT>;
+    constexpr int N = E::kPerVec;
+    constexpr int SEG = 32 * N;
+    extern __shared__ __align__(128) unsigned char cl_smem[];
+    __shared__ ClusterShared sh;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int32_t b = blockIdx.x / kClusterCtas;
+    const bool writer = rank == 0;
+    const int64_t row_bytes = in.V * E::kBytes;
+    const int32_t nseg = (int32_t)((in.V + SEG - 1) / SEG);
+
+    // offsets over max(K_b, 0), clamped to the buffers like the prologue kernel's (every warp, B <= 18)
+    int32_t k_raw = 0;
+    if (lane < in.B) k_raw = in.k_per_row ? in.k_per_row[lane] : in.k_uniform;
+    int64_t incl = k_raw > 0 ? k_raw : 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int64_t up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    const int64_t D = in.n_draft_total;
+    const int64_t excl_b = __shfl_sync(0xffffffffu, incl, b) - (__shfl_sync(0xffffffffu, k_raw, b) > 0 ? __shfl_sync(0xffffffffu, k_raw, b) : 0);
+    const int64_t incl_b = __shfl_sync(0xffffffffu, incl, b);
+    const int32_t kb_raw = __shfl_sync(0xffffffffu, k_raw, b);
+    const int32_t K = kb_raw > 0 ? kb_raw : 0;
+    const int64_t d0 = excl_b < D ? excl_b : D;                   // clamped like off_d[b]
+    const int64_t d1 = incl_b < D ? incl_b : D;                   // off_d[b + 1]
+    const int64_t t0 = d0 + b;
+
+    int status = 0;
+    if (kb_raw < 0 || excl_b + K > D) status |= 1;                // SPECV_ROW_BAD_K
+    const float T = in.temperature[in.per_row_temperature ? b : 0];
+    if (!(T > 0.0f) || isinf(T)) status |= 2;                     // SPECV_ROW_BAD_TEMPERATURE
+    if (K > kClusterMaxK) status |= 16;                           // the host only sends batches that fit
+
+    if (tid == 0) { sh.first_reject = K; sh.bad_token = 0; sh.err = 0; }
+    if (tid < kClusterCtas) sh.err_of[tid] = 0;
+    if (tid == 32) {
+        mbar_init(smem_u32(&sh.bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (!(status & 1)) {
+        for (int32_t i = tid; i < K; i += kClusterThreads) {
+            const int32_t x = in.tokens[d0 + i];
+            if (x < 0 || (int64_t)x >= in.V) sh.bad_token = 1;
+        }
+    }
+    __syncthreads();
+    if (sh.bad_token) status |= 4;                                // SPECV_ROW_BAD_TOKEN
+
+    // slots of this sequence in the packed outputs (clamped offsets: together they tile [0, D + B));
+    // the last cluster also owns the slots no sequence reaches
+    const int64_t slot_end = (b == in.B - 1) ? D + in.B : d1 + b + 1;
+    if (status) {                 // the same in every CTA of the cluster: no barrier is left behind
+        if (writer) {
+            for (int64_t s = t0 + tid; s < slot_end; s += kClusterThreads) emitted[s] = -1;
+            if (tid == 0) {
+                accepted_len[b] = 0;
+                if (row_status) row_status[b] = status;
+                if (next.out) next.out[b] = next_lookahead_of(kb_raw, 0, next.k_min, next.k_max);
+            }
+        }
+        return;
+    }
+
+    // ---- every row's slice into shared memory, all copies in flight at once --------------------------
+    const int32_t n_rows = 2 * K + 1;                             // rows 0..K target, K+1..2K draft
+    const int64_t slice_off = (int64_t)rank * slice_bytes;
+    const int32_t my_bytes = (int32_t)(row_bytes - slice_off < slice_bytes ? (row_bytes - slice_off > 0 ? row_bytes - slice_off : 0)
+                                                                           : slice_bytes);
+    auto row_ptr = [&](int32_t r) {
+        return r <= K ? in.target + (t0 + r) * in.pitch_t : in.draft + (d0 + (r - K - 1)) * in.pitch_d;
+    };
+    volatile int* err = &sh.err;
+    if (my_bytes > 0) {
+        if (warp == 0) {
+            if (lane == 0) mbar_expect_tx(smem_u32(&sh.bar), (uint32_t)my_bytes * (uint32_t)n_rows);
+            __syncwarp();
+            for (int32_t r = lane; r < n_rows; r += 32)
+                bulk_load(smem_u32(cl_smem + (size_t)r * slice_bytes), row_ptr(r) + slice_off, (uint32_t)my_bytes,
+                          smem_u32(&sh.bar));
+        }
+        mbar_wait(smem_u32(&sh.bar), 0, err, 71);
+    }
+    const float c = (float)(kLog2e / (double)T);
+    const int32_t my_vecs = my_bytes / 16;
+
+    // ---- row statistics of the slices: one warp per row ---------------------------------------------
+    for (int32_t r = warp; r < n_rows; r += kClusterWarps) {
+        const uint4* src = reinterpret_cast<const uint4*>(cl_smem + (size_t)r * slice_bytes);
+        float ref = kNoMax, s0 = 0.f, s1 = 0.f;
+        for (int32_t v = lane; v < my_vecs; v += 32 * 2) {
+            uint4 raw[2];
+            raw[0] = src[v];
+            raw[1] = v + 32 < my_vecs ? src[v + 32] : neg_inf_vec(E::kNegInfWord);
+            float x[2 * N];
+            E::unpack(raw[0], x);
+            E::unpack(raw[1], x + N);
+            float mx = x[0];
+#pragma unroll
+            for (int k = 1; k < 2 * N; ++k) mx = fmaxf(mx, x[k]);
+            const float cand = mx * c;
+            if (cand > ref) {
+                const float f = ex2_approx(ref - cand);
+                s0 *= f; s1 *= f;
+                ref = cand;
+            }
+            const unsigned long long cc = pack_f32x2(c, c), nr = pack_f32x2(-ref, -ref);
+            unsigned long long acc = pack_f32x2(s0, s1);
+#pragma unroll
+            for (int k = 0; k < 2 * N; k += 2) {
+                float a0, a1;
+                unpack_f32x2(fma_f32x2(pack_f32x2(x[k], x[k + 1]), cc, nr), a0, a1);
+                acc = add_f32x2(acc, pack_f32x2(ex2_approx(a0), ex2_approx(a1)));
+            }
+            unpack_f32x2(acc, s0, s1);
+        }
+        float sum = s0 + s1;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float oref = __shfl_xor_sync(0xffffffffu, ref, o);
+            const float osum = __shfl_xor_sync(0xffffffffu, sum, o);
+            merge_ref_sum(ref, sum, oref, osum);
+        }
+        // entry [r][rank] of every CTA's table: lanes 0..7 write one CTA each
+        if (lane < kClusterCtas) {
+            const uint32_t dst = map_to_cta(&sh.part[r * kClusterCtas + rank], (uint32_t)lane);
+            asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(dst), "f"(ref), "f"(sum) : "memory");
+        }
+    }
+    if (warp == kClusterWarps - 1 && lane < kClusterCtas) {       // this CTA's copies: arrived or not
+        const uint32_t dst = map_to_cta(&sh.err_of[rank], (uint32_t)lane);
+        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(dst), "r"((uint32_t)*err) : "memory");
+    }
+    cluster_barrier();                                            // #1: all statistics everywhere
+    int any_err = 0;
+#pragma unroll
+    for (int i = 0; i < kClusterCtas; ++i) any_err |= sh.err_of[i];
+    if (any_err) {                // the same in every CTA; nothing more is exchanged
+        if (writer) {
+            for (int64_t s = t0 + tid; s < slot_end; s += kClusterThreads) emitted[s] = -1;
+            if (tid == 0) {
+                accepted_len[b] = 0;
+                if (row_status) row_status[b] = 16 | (any_err << 8);          // SPECV_ROW_INTERNAL
+                if (next.out) next.out[b] = next_lookahead_of(kb_raw, 0, next.k_min, next.k_max);
+            }
+        }
+        if (*err && tid == 0) {   // copies that were issued may still land in this CTA's shared memory
+            const long long t_wait = clock64();
+            while (clock64() - t_wait < 200000) {}
+        }
+        __syncthreads();
+        return;
+    }
+
+    // ---- decisions: every draft position in parallel, in double; first rejection ---------------------
+    for (int32_t i = warp; i < K; i += kClusterWarps) {
+        const RowNorm np = warp_merge_splits(sh.part, i, kClusterCtas, lane);
+        const RowNorm nq = warp_merge_splits(sh.part, K + 1 + i, kClusterCtas, lane);
+        if (lane == 0) {
+            const int32_t x = in.tokens[d0 + i];
+            const double lp = (double)E::load1(in.target + (t0 + i) * in.pitch_t, x);
+            const double lq = (double)E::load1(in.draft + (d0 + i) * in.pitch_d, x);
+            const double p = exp2(lp * (double)c - (double)np.ref) / np.sum;
+            const double q = exp2(lq * (double)c - (double)nq.ref) / nq.sum;
+            if (writer && diag_p) diag_p[d0 + i] = (float)p;
+            if (writer && diag_q) diag_q[d0 + i] = (float)q;
+            const double u = (double)in.uniforms[t0 + i];
+            if (!(u * q < p)) atomicMin(&sh.first_reject, i);
+        }
+    }
+    __syncthreads();
+    const int32_t n = sh.first_reject;
+
+    if (warp == 0) {
+        const RowNorm np = warp_merge_splits(sh.part, n, kClusterCtas, lane);
+        RowNorm nq{0.f, 1.0};
+        if (n < K) nq = warp_merge_splits(sh.part, K + 1 + n, kClusterCtas, lane);
+        if (lane == 0) {
+            SampleRows& rows = sh.rows;
+            rows.p = in.target + (t0 + n) * in.pitch_t;
+            rows.p_aligned = true;                                // the host sends aligned rows only
+            rows.c = c;
+            rows.p_ref = np.ref;
+            rows.q = nullptr; rows.q_aligned = false; rows.q_ref = 0.f; rows.kappa = 0.f;
+            if (n < K) {
+                rows.q = in.draft + (d0 + n) * in.pitch_d;
+                rows.q_aligned = true;
+                rows.q_ref = nq.ref;
+                rows.kappa = (float)(np.sum / nq.sum);
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- segment sums of the drawn-from distribution, from the slices in shared memory ---------------
+    float* const seg = reinterpret_cast<float*>(cl_smem + (size_t)n_rows * slice_bytes);
+    const int32_t seg0 = (int32_t)(slice_off / 512);              // first segment of this CTA's slice
+    const int32_t my_segs = (my_vecs + 31) / 32;
+    auto segment_pass = [&](const SampleRows& sr) {
+        const uint4* sp = reinterpret_cast<const uint4*>(cl_smem + (size_t)n * slice_bytes);
+        const uint4* sq = reinterpret_cast<const uint4*>(cl_smem + (size_t)(K + 1 + (n < K ? n : 0)) * slice_bytes);
+        for (int32_t s = warp; s < my_segs; s += kClusterWarps) {
+            const int32_t v = s * 32 + lane;
+            float a = 0.f;
+            if (v < my_vecs) {
+                float r[N];
+                mass_of_raw<DT>(sr, sp[v], sr.q ? sq[v] : make_uint4(0u, 0u, 0u, 0u), r);
+#pragma unroll
+                for (int k = 0; k < N; ++k) a += r[k];
+            }
+            a = warp_sum(a);
+            if (lane < kClusterCtas) {
+                const uint32_t dst = map_to_cta(&seg[seg0 + s], (uint32_t)lane);
+                asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(dst), "f"(a) : "memory");
+            }
+        }
+        cluster_barrier();
+    };
+    SampleRows sr = sh.rows;
+    segment_pass(sr);                                             // #2
+    if (sr.q && !(warp_segment_total(seg, nseg, lane) > 0.0)) {   // the same table, the same verdict everywhere
+        // the residual rounded to nothing: sample from the target row itself
+        status |= 8;              // SPECV_ROW_ZERO_RESIDUAL
+        sr.q = nullptr;
+        cluster_barrier();        // everyone has read the table before it is rewritten
+        segment_pass(sr);
+    }
+    if (writer) {
+        __shared__ int32_t token_slot;
+        if (warp == 0) {
+            int32_t token = locate_in_segments<DT, true>(sr, in.V, (double)in.uniforms[t0 + K], seg, nseg, lane);
+            if (token < 0) token = (int32_t)(in.V - 1);           // a row without any mass (all logits -inf)
+            if (lane == 0) token_slot = token;
+        }
+        __syncthreads();
+        const int32_t token = token_slot;
+        for (int64_t i = tid; t0 + i < slot_end; i += kClusterThreads)
+            emitted[t0 + i] = (i < n) ? in.tokens[d0 + i] : (i == n ? token : -1);
+        if (tid == 0) {
+            accepted_len[b] = n;
+            if (row_status) row_status[b] = status;
+            if (next.out) next.out[b] = next_lookahead_of(kb_raw, n, next.k_min, next.k_max);
+        }
+    }
+}
+
+}  // namespace specv

@@ -26,11 +26,13 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
-@pytest.fixture(params=["streaming", "ring"])
+@pytest.fixture(params=["streaming", "ring", "cluster"])
 def kernel_path(request):
-    """Runs a GPU test once per kernel set (the ring set falls back to streaming for shapes
-    it does not take, so both parametrisations are always valid)."""
+    """Runs a GPU test once per kernel set (the ring set falls back to streaming, the one-launch
+    cluster form to the automatic choice, for shapes they do not take, so every parametrisation is
+    always valid)."""
     from paper_2411_00853_b200 import binding
-    binding.set_path(binding.PATH_STREAMING if request.param == "streaming" else binding.PATH_RING)
+    binding.set_path({"streaming": binding.PATH_STREAMING, "ring": binding.PATH_RING,
+                      "cluster": binding.PATH_CLUSTER}[request.param])
     yield request.param
     binding.set_path(binding.PATH_AUTO)

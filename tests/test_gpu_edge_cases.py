@@ -17,6 +17,8 @@ ZERO_RESIDUAL = binding.ROW_ZERO_RESIDUAL
 
 
 def _expect_path(kernel_path, ring_capable=True):
+    if kernel_path == "cluster":
+        return                  # taken where the batch fits a cluster per sequence, else the automatic choice
     want = binding.PATH_RING if (kernel_path == "ring" and ring_capable) else binding.PATH_STREAMING
     assert binding.last_path() == want
 

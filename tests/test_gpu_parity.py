@@ -26,7 +26,8 @@ def test_hand_cases(kernel_path, case):
     w = _Case(*hand_case_inputs(case))
     acc, em, st, dp, dq = DeviceBatch(w).run()
     assert acc[0] == case["expect_len"] and em.tolist() == case["expect_emitted"] and st[0] == 0
-    assert binding.last_path() == (binding.PATH_RING if kernel_path == "ring" else binding.PATH_STREAMING)
+    if kernel_path != "cluster":          # the cluster form takes the cases whose rows are whole 16-byte vectors
+        assert binding.last_path() == (binding.PATH_RING if kernel_path == "ring" else binding.PATH_STREAMING)
     if "expect_ptok" in case:
         np.testing.assert_allclose(dp, case["expect_ptok"], rtol=1e-5)
         np.testing.assert_allclose(dq, case["expect_qtok"], rtol=1e-5)
@@ -173,7 +174,8 @@ def test_argument_errors_come_back_as_status_codes():
                                   k_max, next_k)
 
     assert call_ex(0) == 0 and call_ex(binding.FLAG_RING | binding.FLAG_EARLY_EXIT) == 0
-    assert call_ex(binding.FLAG_RING | binding.FLAG_STREAMING) == 9 and call_ex(8) == 9 and call_ex(1 << 31) == 9
+    assert call_ex(binding.FLAG_RING | binding.FLAG_STREAMING) == 9 and call_ex(16) == 9 and call_ex(1 << 31) == 9
+    assert call_ex(binding.FLAG_CLUSTER) == 0 and call_ex(binding.FLAG_CLUSTER | binding.FLAG_RING) == 9
     nk = torch.zeros(2, dtype=torch.int32, device="cuda")
     assert call_ex(0, 1, 8, nk.data_ptr()) == 0
     assert call_ex(0, -1, 8, nk.data_ptr()) == 2 and call_ex(0, 5, 4, nk.data_ptr()) == 2
@@ -187,14 +189,17 @@ def test_kernel_set_selection(kernel_path):
     fall-back), and shapes they cannot take go to the streaming kernels."""
     w = W.make_config(5, B=12, V=32000)
     DeviceBatch(w).run()
-    assert binding.last_path() == (binding.PATH_RING if kernel_path == "ring" else binding.PATH_STREAMING)
+    assert binding.last_path() == {"ring": binding.PATH_RING, "streaming": binding.PATH_STREAMING,
+                                   "cluster": binding.PATH_RING}[kernel_path]     # 100 draft rows: too many for the cluster form
     for V in (4099, 31):                       # rows that are not whole 16-byte vectors
         DeviceBatch(W.make_config(5, B=4, V=V)).run()
         assert binding.last_path() == binding.PATH_STREAMING
     DeviceBatch(w, elem_offset=3).run()        # unaligned rows
     assert binding.last_path() == binding.PATH_STREAMING
     binding.set_path(binding.PATH_AUTO)
-    DeviceBatch(W.make_config(1)).run()        # 5 work items: too few for one CTA per item
+    DeviceBatch(W.make_config(1)).run()        # one sequence whose rows fit a cluster's shared memory
+    assert binding.last_path() == binding.PATH_CLUSTER
+    DeviceBatch(W.make_config(1, V=200000)).run()        # 9 rows of 800 KB do not: 5 work items, streaming kernels
     assert binding.last_path() == binding.PATH_STREAMING
     DeviceBatch(W.make_config(5, B=64, V=32000)).run()
     assert binding.last_path() == binding.PATH_RING
