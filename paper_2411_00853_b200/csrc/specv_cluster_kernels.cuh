@@ -18,7 +18,7 @@
 // barrier; the one bounded wait is for the CTA's own copies.
 //
 // Same arithmetic as the streaming kernels: statistics merged per row in double in a fixed order
-// (warp_merge_splits over the eight partials), decisions u q < p in double, masses by mass_of_raw,
+// (warp_merge_splits over the 32 partials of a row), decisions u q < p in double, masses by mass_of_raw,
 // inverse CDF by locate_in_segments.
 #pragma once
 
@@ -32,13 +32,20 @@ constexpr int kClusterWarps = kClusterThreads / 32;
 constexpr int kClusterMaxK = 32;                          // lookahead the shared-memory tables are sized for
 constexpr int kClusterMaxRows = 2 * kClusterMaxK + 1;
 constexpr int kClusterMaxSeqs = 18;                       // 8 CTAs each on 148 SMs; offsets are scanned by one warp
+constexpr int kClusterSub = 4;                            // a CTA's slice of a row is summed in four parts (all warps busy)
+constexpr int kClusterParts = kClusterCtas * kClusterSub; // partial statistics per row: one per lane of the merging warp
 
 struct ClusterShared {
-    float2 part[kClusterMaxRows * kClusterCtas];          // [row][cta]: partial (ref, sum) of every row from every CTA
+    float2 part[kClusterMaxRows * kClusterParts];         // [row][cta][sub]: partial (ref, sum) of every row from every CTA
+    double norm_sum[kClusterMaxRows];                     // merged statistics of every row (each CTA merges for itself)
+    float norm_ref[kClusterMaxRows];
     int err_of[kClusterCtas];                             // a CTA whose copies did not arrive reports here, everywhere
     unsigned long long bar;
     SampleRows rows;
-    int32_t first_reject, bad_token, err;
+    int32_t first_reject, bad_token, err, token;
+    // what the decisions need of every draft position, fetched while the rows are on their way
+    int32_t tok[kClusterMaxK];
+    float lp[kClusterMaxK], lq[kClusterMaxK], u[kClusterMaxK + 1];
 };
 
 __device__ __forceinline__ uint32_t map_to_cta(const void* smem_ptr, uint32_t cta) {
@@ -97,19 +104,48 @@ specv_cluster_pass(BatchView in, int32_t slice_bytes, int32_t* __restrict__ acce
 
     if (tid == 0) { sh.first_reject = K; sh.bad_token = 0; sh.err = 0; }
     if (tid < kClusterCtas) sh.err_of[tid] = 0;
-    if (tid == 32) {
-        mbar_init(smem_u32(&sh.bar), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
     __syncthreads();
-    if (!(status & 1)) {
-        for (int32_t i = tid; i < K; i += kClusterThreads) {
-            const int32_t x = in.tokens[d0 + i];
-            if (x < 0 || (int64_t)x >= in.V) sh.bad_token = 1;
+
+    // ---- every row's slice into shared memory, all copies in flight at once: issued first, everything
+    // else the pass needs from global memory is fetched while they are on their way --------------------
+    const int32_t n_rows = 2 * K + 1;                             // rows 0..K target, K+1..2K draft
+    const int64_t slice_off = (int64_t)rank * slice_bytes;
+    const int32_t my_bytes = (int32_t)(row_bytes - slice_off < slice_bytes ? (row_bytes - slice_off > 0 ? row_bytes - slice_off : 0)
+                                                                           : slice_bytes);
+    auto row_ptr = [&](int32_t r) {
+        return r <= K ? in.target + (t0 + r) * in.pitch_t : in.draft + (d0 + (r - K - 1)) * in.pitch_d;
+    };
+    volatile int* err = &sh.err;
+    const bool copying = !status && my_bytes > 0;                 // the same in every warp
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_init(smem_u32(&sh.bar), 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            if (copying) mbar_expect_tx(smem_u32(&sh.bar), (uint32_t)my_bytes * (uint32_t)n_rows);
+        }
+        __syncwarp();
+        if (copying)
+            for (int32_t r = lane; r < n_rows; r += 32)
+                bulk_load(smem_u32(cl_smem + (size_t)r * slice_bytes), row_ptr(r) + slice_off, (uint32_t)my_bytes,
+                          smem_u32(&sh.bar));
+    }
+    // the drafted tokens, their two logits and the uniforms (one thread per position)
+    if (!(status & (1 | 16))) {
+        for (int32_t i = tid; i <= K; i += kClusterThreads) {
+            sh.u[i] = in.uniforms[t0 + i];
+            if (i < K) {
+                const int32_t x = in.tokens[d0 + i];
+                const bool ok = x >= 0 && (int64_t)x < in.V;
+                if (!ok) sh.bad_token = 1;
+                sh.tok[i] = x;
+                sh.lp[i] = ok ? E::load1(in.target + (t0 + i) * in.pitch_t, x) : 0.f;
+                sh.lq[i] = ok ? E::load1(in.draft + (d0 + i) * in.pitch_d, x) : 0.f;
+            }
         }
     }
     __syncthreads();
     if (sh.bad_token) status |= 4;                                // SPECV_ROW_BAD_TOKEN
+    if (copying) mbar_wait(smem_u32(&sh.bar), 0, err, 71);        // also before giving up on a bad token: the copies target this CTA
 
     // slots of this sequence in the packed outputs (clamped offsets: together they tile [0, D + B));
     // the last cluster also owns the slots no sequence reaches
@@ -125,37 +161,20 @@ specv_cluster_pass(BatchView in, int32_t slice_bytes, int32_t* __restrict__ acce
         }
         return;
     }
-
-    // ---- every row's slice into shared memory, all copies in flight at once --------------------------
-    const int32_t n_rows = 2 * K + 1;                             // rows 0..K target, K+1..2K draft
-    const int64_t slice_off = (int64_t)rank * slice_bytes;
-    const int32_t my_bytes = (int32_t)(row_bytes - slice_off < slice_bytes ? (row_bytes - slice_off > 0 ? row_bytes - slice_off : 0)
-                                                                           : slice_bytes);
-    auto row_ptr = [&](int32_t r) {
-        return r <= K ? in.target + (t0 + r) * in.pitch_t : in.draft + (d0 + (r - K - 1)) * in.pitch_d;
-    };
-    volatile int* err = &sh.err;
-    if (my_bytes > 0) {
-        if (warp == 0) {
-            if (lane == 0) mbar_expect_tx(smem_u32(&sh.bar), (uint32_t)my_bytes * (uint32_t)n_rows);
-            __syncwarp();
-            for (int32_t r = lane; r < n_rows; r += 32)
-                bulk_load(smem_u32(cl_smem + (size_t)r * slice_bytes), row_ptr(r) + slice_off, (uint32_t)my_bytes,
-                          smem_u32(&sh.bar));
-        }
-        mbar_wait(smem_u32(&sh.bar), 0, err, 71);
-    }
     const float c = (float)(kLog2e / (double)T);
     const int32_t my_vecs = my_bytes / 16;
 
-    // ---- row statistics of the slices: one warp per row ---------------------------------------------
-    for (int32_t r = warp; r < n_rows; r += kClusterWarps) {
+    // ---- row statistics of the slices: a warp per (row, quarter of the slice) ------------------------
+    for (int32_t item = warp; item < n_rows * kClusterSub; item += kClusterWarps) {
+        const int32_t r = item / kClusterSub, sub = item % kClusterSub;
         const uint4* src = reinterpret_cast<const uint4*>(cl_smem + (size_t)r * slice_bytes);
+        const int32_t v_begin = (int32_t)((int64_t)my_vecs * sub / kClusterSub);
+        const int32_t v_end = (int32_t)((int64_t)my_vecs * (sub + 1) / kClusterSub);
         float ref = kNoMax, s0 = 0.f, s1 = 0.f;
-        for (int32_t v = lane; v < my_vecs; v += 32 * 2) {
+        for (int32_t v = v_begin + lane; v < v_end; v += 32 * 2) {
             uint4 raw[2];
             raw[0] = src[v];
-            raw[1] = v + 32 < my_vecs ? src[v + 32] : neg_inf_vec(E::kNegInfWord);
+            raw[1] = v + 32 < v_end ? src[v + 32] : neg_inf_vec(E::kNegInfWord);
             float x[2 * N];
             E::unpack(raw[0], x);
             E::unpack(raw[1], x + N);
@@ -185,9 +204,9 @@ specv_cluster_pass(BatchView in, int32_t slice_bytes, int32_t* __restrict__ acce
             const float osum = __shfl_xor_sync(0xffffffffu, sum, o);
             merge_ref_sum(ref, sum, oref, osum);
         }
-        // entry [r][rank] of every CTA's table: lanes 0..7 write one CTA each
+        // entry [r][rank][sub] of every CTA's table: lanes 0..7 write one CTA each
         if (lane < kClusterCtas) {
-            const uint32_t dst = map_to_cta(&sh.part[r * kClusterCtas + rank], (uint32_t)lane);
+            const uint32_t dst = map_to_cta(&sh.part[r * kClusterParts + rank * kClusterSub + sub], (uint32_t)lane);
             asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(dst), "f"(ref), "f"(sum) : "memory");
         }
     }
@@ -216,42 +235,34 @@ specv_cluster_pass(BatchView in, int32_t slice_bytes, int32_t* __restrict__ acce
         return;
     }
 
-    // ---- decisions: every draft position in parallel, in double; first rejection ---------------------
-    for (int32_t i = warp; i < K; i += kClusterWarps) {
-        const RowNorm np = warp_merge_splits(sh.part, i, kClusterCtas, lane);
-        const RowNorm nq = warp_merge_splits(sh.part, K + 1 + i, kClusterCtas, lane);
-        if (lane == 0) {
-            const int32_t x = in.tokens[d0 + i];
-            const double lp = (double)E::load1(in.target + (t0 + i) * in.pitch_t, x);
-            const double lq = (double)E::load1(in.draft + (d0 + i) * in.pitch_d, x);
-            const double p = exp2(lp * (double)c - (double)np.ref) / np.sum;
-            const double q = exp2(lq * (double)c - (double)nq.ref) / nq.sum;
-            if (writer && diag_p) diag_p[d0 + i] = (float)p;
-            if (writer && diag_q) diag_q[d0 + i] = (float)q;
-            const double u = (double)in.uniforms[t0 + i];
-            if (!(u * q < p)) atomicMin(&sh.first_reject, i);
-        }
+    // ---- every row's statistics merged (a warp per row, double, fixed order), then the decisions: every
+    // draft position in parallel, in double; first rejection ------------------------------------------
+    for (int32_t r = warp; r < n_rows; r += kClusterWarps) {
+        const RowNorm nr = warp_merge_splits(sh.part, r, kClusterParts, lane);
+        if (lane == 0) { sh.norm_ref[r] = nr.ref; sh.norm_sum[r] = nr.sum; }
+    }
+    __syncthreads();
+    for (int32_t i = tid; i < K; i += kClusterThreads) {
+        const double p = exp2((double)sh.lp[i] * (double)c - (double)sh.norm_ref[i]) / sh.norm_sum[i];
+        const double q = exp2((double)sh.lq[i] * (double)c - (double)sh.norm_ref[K + 1 + i]) / sh.norm_sum[K + 1 + i];
+        if (writer && diag_p) diag_p[d0 + i] = (float)p;
+        if (writer && diag_q) diag_q[d0 + i] = (float)q;
+        if (!((double)sh.u[i] * q < p)) atomicMin(&sh.first_reject, i);
     }
     __syncthreads();
     const int32_t n = sh.first_reject;
-
-    if (warp == 0) {
-        const RowNorm np = warp_merge_splits(sh.part, n, kClusterCtas, lane);
-        RowNorm nq{0.f, 1.0};
-        if (n < K) nq = warp_merge_splits(sh.part, K + 1 + n, kClusterCtas, lane);
-        if (lane == 0) {
-            SampleRows& rows = sh.rows;
-            rows.p = in.target + (t0 + n) * in.pitch_t;
-            rows.p_aligned = true;                                // the host sends aligned rows only
-            rows.c = c;
-            rows.p_ref = np.ref;
-            rows.q = nullptr; rows.q_aligned = false; rows.q_ref = 0.f; rows.kappa = 0.f;
-            if (n < K) {
-                rows.q = in.draft + (d0 + n) * in.pitch_d;
-                rows.q_aligned = true;
-                rows.q_ref = nq.ref;
-                rows.kappa = (float)(np.sum / nq.sum);
-            }
+    if (tid == 0) {
+        SampleRows& rows = sh.rows;
+        rows.p = in.target + (t0 + n) * in.pitch_t;
+        rows.p_aligned = true;                                    // the host sends aligned rows only
+        rows.c = c;
+        rows.p_ref = sh.norm_ref[n];
+        rows.q = nullptr; rows.q_aligned = false; rows.q_ref = 0.f; rows.kappa = 0.f;
+        if (n < K) {
+            rows.q = in.draft + (d0 + n) * in.pitch_d;
+            rows.q_aligned = true;
+            rows.q_ref = sh.norm_ref[K + 1 + n];
+            rows.kappa = (float)(sh.norm_sum[n] / sh.norm_sum[K + 1 + n]);
         }
     }
     __syncthreads();
@@ -289,17 +300,36 @@ specv_cluster_pass(BatchView in, int32_t slice_bytes, int32_t* __restrict__ acce
         cluster_barrier();        // everyone has read the table before it is rewritten
         segment_pass(sr);
     }
+    // ---- CTA 0 locates the token: prefix over the table, then the crossing segment's vectors straight
+    // from the shared memory of the CTA that holds them ---------------------------------------------
     if (writer) {
-        __shared__ int32_t token_slot;
         if (warp == 0) {
-            int32_t token = locate_in_segments<DT, true>(sr, in.V, (double)in.uniforms[t0 + K], seg, nseg, lane);
+            const int32_t row_p = n, row_q = K + 1 + (n < K ? n : 0);
+            auto slice_vector = [&](int32_t row, int64_t v) -> uint4 {
+                const int64_t byte = v * 16;
+                if (byte >= row_bytes) return neg_inf_vec(E::kNegInfWord);
+                const uint32_t owner = (uint32_t)(byte / slice_bytes);
+                const uint32_t a = map_to_cta(cl_smem + (size_t)row * slice_bytes + (size_t)(byte - (int64_t)owner * slice_bytes), owner);
+                uint4 r;
+                asm volatile("ld.shared::cluster.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(a) : "memory");
+                return r;
+            };
+            int32_t token = locate_in_segments_with<DT>(sr, (double)sh.u[K], seg, nseg, lane,
+                                                        [&](int64_t v, uint4& rawp, uint4& rawq) {
+                                                            rawp = slice_vector(row_p, v);
+                                                            rawq = sr.q ? slice_vector(row_q, v) : make_uint4(0u, 0u, 0u, 0u);
+                                                        });
             if (token < 0) token = (int32_t)(in.V - 1);           // a row without any mass (all logits -inf)
-            if (lane == 0) token_slot = token;
+            if (lane == 0) sh.token = token;
         }
         __syncthreads();
-        const int32_t token = token_slot;
+    }
+    cluster_barrier();            // nobody's shared memory goes away while CTA 0 may still read it
+    if (writer) {
+        const int32_t token = sh.token;
         for (int64_t i = tid; t0 + i < slot_end; i += kClusterThreads)
-            emitted[t0 + i] = (i < n) ? in.tokens[d0 + i] : (i == n ? token : -1);
+            emitted[t0 + i] = (i < n) ? sh.tok[i] : (i == n ? token : -1);
         if (tid == 0) {
             accepted_len[b] = n;
             if (row_status) row_status[b] = status;

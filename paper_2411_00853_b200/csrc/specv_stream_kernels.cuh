@@ -304,18 +304,15 @@ __device__ __forceinline__ void mass_of_raw(const SampleRows& sr, const uint4& r
 // the segment where the running mass first exceeds u * total, then the token inside it
 // (its vectors are re-read and their masses recomputed exactly as for the segment sums).
 // Returns the token to every lane, or -1 if the total mass is 0.
-template <int DT, bool FAST>
-__device__ int32_t locate_in_segments(const SampleRows& sr, int64_t V, double u, const float* seg,
-                                      int32_t nseg, int lane) {
+// `load_pair(v, rawp, rawq)` supplies 16-byte vector v of the row(s) the masses are taken from.
+template <int DT, class LoadPair>
+__device__ int32_t locate_in_segments_with(const SampleRows& sr, double u, const float* seg, int32_t nseg, int lane,
+                                           LoadPair load_pair) {
     using E = Elt<DT>;
     constexpr int N = E::kPerVec;
-    auto load = [&](const char* row, bool aligned, int64_t v) -> uint4 {
-        if (FAST) return v * N < V ? ld_stream16(row + v * 16) : neg_inf_vec(E::kNegInfWord);
-        return load_vec<DT>(row, aligned, v, V);
-    };
     auto masses = [&](int64_t v, float* r) {
-        const uint4 rawp = load(sr.p, sr.p_aligned, v);
-        const uint4 rawq = sr.q ? load(sr.q, sr.q_aligned, v) : make_uint4(0u, 0u, 0u, 0u);
+        uint4 rawp, rawq;
+        load_pair(v, rawp, rawq);
         mass_of_raw<DT>(sr, rawp, rawq, r);
     };
     const int32_t per = (nseg + 31) / 32;
@@ -371,6 +368,22 @@ __device__ int32_t locate_in_segments(const SampleRows& sr, int64_t V, double u,
         token = (int32_t)(((int64_t)found_seg * 32 + src) * N + __shfl_sync(0xffffffffu, k_sel, src));
     }
     return token;
+}
+
+// The same with the vectors read from the rows in global memory.
+template <int DT, bool FAST>
+__device__ int32_t locate_in_segments(const SampleRows& sr, int64_t V, double u, const float* seg,
+                                      int32_t nseg, int lane) {
+    using E = Elt<DT>;
+    constexpr int N = E::kPerVec;
+    auto load = [&](const char* row, bool aligned, int64_t v) -> uint4 {
+        if (FAST) return v * N < V ? ld_stream16(row + v * 16) : neg_inf_vec(E::kNegInfWord);
+        return load_vec<DT>(row, aligned, v, V);
+    };
+    return locate_in_segments_with<DT>(sr, u, seg, nseg, lane, [&](int64_t v, uint4& rawp, uint4& rawq) {
+        rawp = load(sr.p, sr.p_aligned, v);
+        rawq = sr.q ? load(sr.q, sr.q_aligned, v) : make_uint4(0u, 0u, 0u, 0u);
+    });
 }
 
 // Segment masses of the distribution `sr` describes into seg[] (shared, one float per 32-vector
