@@ -35,8 +35,8 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
 # kernel from the ncu capture summarised under profiles/; only valid for the kernel source
 # it was taken from (sha256 of the files that kernel is compiled from), otherwise reported as null.
-NCU_TRAFFIC = {"csrc_sha256": "b39e20532d800f3a2bfe461818343381e018b694d731356f3c6fe4dc3127ceea",
-               "workload": "config3 capture of specv_ring_stats (279.14 MB read + 4.20 MB written for 279.09 MB of logits) scaled by logit bytes to config5", "bytes_per_launch": 2425103345}
+NCU_TRAFFIC = {"csrc_sha256": "1e214ecf62836d7d13fa6d3a5675307fc503a6c3f67182c204e3c336a43bbe13",
+               "workload": "config3 capture of specv_ring_stats (279.14 MB read + 4.14 MB written for 279.09 MB of logits) scaled by logit bytes to config5", "bytes_per_launch": 2424588446}
 
 
 # kernel set of a pass as spec_verify_last_path reports it
