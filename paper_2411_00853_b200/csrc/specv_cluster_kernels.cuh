@@ -293,13 +293,6 @@ specv_cluster_pass(BatchView in, int32_t slice_bytes, int32_t* __restrict__ acce
     };
     SampleRows sr = sh.rows;
     segment_pass(sr);                                             // #2
-    if (sr.q && !(warp_segment_total(seg, nseg, lane) > 0.0)) {   // the same table, the same verdict everywhere
-        // the residual rounded to nothing: sample from the target row itself
-        status |= 8;              // SPECV_ROW_ZERO_RESIDUAL
-        sr.q = nullptr;
-        cluster_barrier();        // everyone has read the table before it is rewritten
-        segment_pass(sr);
-    }
     // ---- CTA 0 locates the token: prefix over the table, then the crossing segment's vectors straight
     // from the shared memory of the CTA that holds them ---------------------------------------------
     if (writer) {
@@ -315,18 +308,28 @@ specv_cluster_pass(BatchView in, int32_t slice_bytes, int32_t* __restrict__ acce
                              : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(a) : "memory");
                 return r;
             };
-            int32_t token = locate_in_segments_with<DT>(sr, (double)sh.u[K], seg, nseg, lane,
-                                                        [&](int64_t v, uint4& rawp, uint4& rawq) {
-                                                            rawp = slice_vector(row_p, v);
-                                                            rawq = sr.q ? slice_vector(row_q, v) : make_uint4(0u, 0u, 0u, 0u);
-                                                        });
-            if (token < 0) token = (int32_t)(in.V - 1);           // a row without any mass (all logits -inf)
+            const int32_t token = locate_in_segments_with<DT>(sr, (double)sh.u[K], seg, nseg, lane,
+                                                              [&](int64_t v, uint4& rawp, uint4& rawq) {
+                                                                  rawp = slice_vector(row_p, v);
+                                                                  rawq = sr.q ? slice_vector(row_q, v) : make_uint4(0u, 0u, 0u, 0u);
+                                                              });
             if (lane == 0) sh.token = token;
         }
         __syncthreads();
-    }
-    cluster_barrier();            // nobody's shared memory goes away while CTA 0 may still read it
-    if (writer) {
+        if (sh.token < 0 && sr.q) {       // block-uniform; rare
+            // the residual rounded to nothing: sample from the target row itself.  This CTA alone, the row
+            // read from global memory (the other CTAs have nothing more to contribute)
+            status |= 8;                  // SPECV_ROW_ZERO_RESIDUAL
+            sr.q = nullptr;
+            block_segment_sums<DT, kClusterWarps, true>(sr, in.V, seg, warp, [] { __syncthreads(); });
+            if (warp == 0) {
+                const int32_t token = locate_in_segments<DT, true>(sr, in.V, (double)sh.u[K], seg, nseg, lane);
+                if (lane == 0) sh.token = token;
+            }
+            __syncthreads();
+        }
+        if (tid == 0 && sh.token < 0) sh.token = (int32_t)(in.V - 1);     // a row without any mass (all logits -inf)
+        __syncthreads();
         const int32_t token = sh.token;
         for (int64_t i = tid; t0 + i < slot_end; i += kClusterThreads)
             emitted[t0 + i] = (i < n) ? sh.tok[i] : (i == n ? token : -1);
@@ -336,6 +339,7 @@ specv_cluster_pass(BatchView in, int32_t slice_bytes, int32_t* __restrict__ acce
             if (next.out) next.out[b] = next_lookahead_of(kb_raw, n, next.k_min, next.k_max);
         }
     }
+    cluster_barrier();            // nobody's shared memory goes away while CTA 0 may still read it
 }
 
 }  // namespace specv
